@@ -1,0 +1,443 @@
+#!/usr/bin/env python
+"""Benchmark of the hot path: importance-weighted group-advantage PG loss, forward + backward.
+
+A "step" is one pass of the whole path (row statistics, finalize, dlogits) over one synthetic
+mini-batch of the SLM shape: 8 prompts x 8 generations, responses of 256-1024 tokens padded to
+1024 and masked, V = 151936, bf16 logits.  The metric is unmasked tokens per second.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+N > 1 is launched with torch.distributed.run, one rank per GPU; every rank runs its own
+mini-batch (the path partitions by prompt group, so there is no collective on the data path:
+weak scaling) and the time is the maximum over ranks.
+
+--impl reference times the float64 CPU oracle, as it stands, on the host cores (the paper ships
+no implementation to run); each of its steps is a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2510_03515_b200 import synth  # noqa: E402
+
+METRIC = "PG loss fwd+bwd tokens/sec at V=151936 bf16"
+UNIT = "tokens/s"
+WORKLOAD = "slm"
+
+
+# ------------------------------------------------------------------------------------------------
+# helpers
+# ------------------------------------------------------------------------------------------------
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons for one GPU while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.rows = []
+        self.proc = None
+        self.thread = None
+        try:
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            self.gpu_id = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
+        except Exception:
+            self.gpu_id = str(device_index)
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu_id}", f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._pump, daemon=True)
+        self.thread.start()
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons, power = [], [], set(), []
+        for ts, line in self.rows:
+            if ts < t0 or ts > t1 + 0.1:
+                continue
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+                power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                  "sw_power_cap"), parts[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def torch_token_logp(logits: torch.Tensor, targets: torch.Tensor, rows_per_block: int = 2048):
+    """'Current' log-probs used only to synthesise the behaviour policy's stored log-probs
+    (input generation with library ops; not part of the measured path)."""
+    out = torch.empty(logits.shape[0], dtype=torch.float32, device=logits.device)
+    for r0 in range(0, logits.shape[0], rows_per_block):
+        z = logits[r0:r0 + rows_per_block].float()
+        lse = torch.logsumexp(z, dim=1)
+        zy = z.gather(1, targets[r0:r0 + rows_per_block].long().unsqueeze(1)).squeeze(1)
+        out[r0:r0 + rows_per_block] = zy - lse
+    return out
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle timing (cpu_baseline leg and --impl reference)
+# ------------------------------------------------------------------------------------------------
+
+def oracle_sample(w: synth.Workload, target_seconds: float = 10.0):
+    """Time the oracle, as it stands, on a bounded sample of the workload: whole groups of the
+    same vocabulary and dtype with proportionally shorter generations.  Returns a dict."""
+    import numpy as np
+
+    import oracle
+    cores = oracle.max_threads()
+
+    def run(seq_len: int):
+        ws = w.scaled(n_prompts=1, seq_len=seq_len, len_lo=max(1, w.len_lo * seq_len // w.seq_len))
+        b = synth.make_batch(ws)
+        bits = synth.bits_numpy(b["logits"])
+        tg, mk = b["targets"].numpy(), b["mask"].numpy()
+        behav = b["behav_noise"].numpy() - 10.0
+        t0 = time.perf_counter()
+        o = oracle.pg_loss(bits, ws.n_seq, ws.seq_len, ws.vocab, tg, mk, behav, b["rewards"].numpy(),
+                           b["group_offsets"].numpy(), 2.0, 0, want_dlogits=False)
+        blk = 128
+        for r0 in range(0, ws.n_rows, blk):  # step 6 in blocks so the float64 rows fit in memory
+            rows = np.arange(r0, min(r0 + blk, ws.n_rows), dtype=np.int64)
+            oracle.dlogits_rows(bits, ws.vocab, ws.seq_len, tg, o["row_ok"], o["lse"], o["coef"], rows)
+        dt = time.perf_counter() - t0
+        return dt, int(o["n_tokens"]), ws
+
+    dt, ntok, ws = run(16)
+    seq_len = int(min(w.seq_len, max(16, 16 * target_seconds / max(dt, 1e-3))))
+    seq_len = max(16, min(seq_len, w.seq_len))
+    dt, ntok, ws = run(seq_len)
+    return {"value": ntok / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{ws.n_seq} generations x {ws.seq_len} padded tokens ({ntok} unmasked), "
+                      f"V={ws.vocab} {ws.dtype}, float64 steps 1-6, {dt:.2f} s",
+            "seconds": dt, "tokens": ntok}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = synth.CONFIGS[WORKLOAD]
+    for _ in range(max(0, min(args.warmup, 1))):
+        oracle_sample(w, target_seconds=1.0)
+    steps = max(1, min(args.steps, 3))
+    tot_tok, tot_s, last = 0, 0.0, None
+    for _ in range(steps):
+        last = oracle_sample(w, target_seconds=8.0)
+        tot_tok += last["tokens"]
+        tot_s += last["seconds"]
+    value = tot_tok / tot_s
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * tot_s / steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": WORKLOAD + " (bounded sample per step)", "vocab": w.vocab,
+                   "logits_dtype": w.dtype},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": last["cores"], "kind": "oracle",
+                         "sample": last["sample"]},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------
+# the CUDA path
+# ------------------------------------------------------------------------------------------------
+
+def run_ours(args):
+    from paper_2510_03515_b200 import binding as rb
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    rb.lib()
+
+    w = synth.CONFIGS[WORKLOAD].scaled(seed=synth.CONFIGS[WORKLOAD].seed + 1000 * rank)
+    if args.seq_len:
+        w = w.scaled(seq_len=args.seq_len, len_lo=max(1, args.seq_len // 4))
+    tok = synth.make_tokens(w)
+    T, V, N = w.n_rows, w.vocab, w.n_seq
+    esize = 2 if w.dtype == "bf16" else 4
+    logits = synth.logits_for_sequences(w, tok["targets"], 0, N, device=dev)
+    targets, mask = tok["targets"].to(dev), tok["mask"].to(dev)
+    rewards, go = tok["rewards"].to(dev), tok["group_offsets"].to(dev)
+    behav = (torch_token_logp(logits, targets) + tok["behav_noise"].to(dev)).contiguous()
+    dlogits = torch.empty_like(logits)
+    desc = rb.make_desc(N, w.seq_len, V, w.n_prompts, logits.dtype, logits.stride(0), 2.0, 0)
+    ws = rb.alloc_workspace(desc, dev)
+    loss = torch.zeros(1, device=dev)
+    token_logp = torch.empty(T, device=dev)
+    adv = torch.empty(N, device=dev)
+    stats = rb.alloc_stats(dev)
+    n_tokens = int(tok["mask"].sum().item())
+
+    def step(ev=None):
+        if ev:
+            ev[0].record()
+        rb.rapid_pg_stats_chunk(desc, logits, 0, T, targets, mask, ws)
+        if ev:
+            ev[1].record()
+        rb.rapid_pg_finalize(desc, behav, rewards, go, loss, token_logp, adv, stats, ws)
+        if ev:
+            ev[2].record()
+        rb.rapid_pg_dlogits_chunk(desc, logits, dlogits, 0, T, targets, ws)
+        if ev:
+            ev[3].record()
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    st = rb.read_stats(stats)
+    live_rows = None
+    # rows pass 2 really streams: unmasked rows of generations with a non-zero coefficient
+    coef_live = (adv != 0).repeat_interleave(w.seq_len)
+    live_rows = int((coef_live & (mask != 0)).sum().item())
+
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    if dist:
+        dist.barrier()
+    torch.cuda.synchronize()
+    if sampler:
+        sampler.start()
+        time.sleep(0.25)
+    t0w = time.time()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for k in range(args.steps):
+        step(evs[k])
+    end.record()
+    torch.cuda.synchronize()
+    t1w = time.time()
+    if dist:
+        dist.barrier()
+    clocks = sampler.stop(t0w, t1w) if sampler else None
+    elapsed_ms = start.elapsed_time(end)
+    if dist:
+        t = torch.tensor([elapsed_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+        tk = torch.tensor([n_tokens], device=dev, dtype=torch.float64)
+        dist.all_reduce(tk, op=dist.ReduceOp.SUM)
+        total_tokens = float(tk.item())
+    else:
+        total_tokens = float(n_tokens)
+    ms_per_step = elapsed_ms / args.steps
+    value = total_tokens / (ms_per_step * 1e-3)
+
+    p1 = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)
+    fin = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)
+    p2 = statistics.mean(e[2].elapsed_time(e[3]) for e in evs)
+    peak, peak_kind = load_peaks()
+    row_bytes = V * esize
+    # algorithmic bytes: pass 1 reads every unmasked row once; pass 2 re-reads the live rows and
+    # writes every row (zeros for the rest)
+    bytes_p1 = n_tokens * row_bytes
+    bytes_p2 = live_rows * row_bytes + T * row_bytes
+    ach_p1 = bytes_p1 / (p1 * 1e-3) / 1e9
+    ach_p2 = bytes_p2 / (p2 * 1e-3) / 1e9
+    ach_all = (bytes_p1 + bytes_p2) / (ms_per_step * 1e-3) / 1e9
+
+    # ---- end to end through the public call with HOST buffers ------------------------------------
+    e2e = None
+    if rank == 0 or dist:
+        e2e = run_e2e(rb, args, desc, w, logits, tok, behav, dlogits, ws, loss, token_logp, adv, stats,
+                      n_tokens, dev, dist)
+
+    if rank != 0:
+        if dist:
+            dist.destroy_process_group()
+        return
+    cpu = oracle_sample(w, target_seconds=10.0) if world == 1 or rank == 0 else None
+    for k in ("seconds", "tokens"):
+        cpu.pop(k, None)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "prompts": w.n_prompts, "generations_per_prompt": w.group_size,
+                   "padded_len": w.seq_len, "vocab": V, "logits_dtype": w.dtype,
+                   "unmasked_tokens_per_gpu": n_tokens, "rows_per_gpu": T,
+                   "l2_policy": f"inputs larger than L2 ({T * row_bytes / 1e9:.1f} GB logits per step)",
+                   "eta": 2.0, "parallelism": f"dp{world} (by prompt group, no data-path collective)"},
+        "clocks": clocks,
+        "e2e": e2e,
+        "gpu_launches": 4 * args.steps,
+        "roofline": {"bound": "hbm", "kernel": "dlogits_kernel (pass 2)", "achieved": ach_p2,
+                     "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": ach_p2 / peak,
+                     "frac_of_8TBs_nominal": ach_p2 / 8000.0, "ms_per_launch": p2,
+                     "algorithmic_bytes_per_launch": bytes_p2, "traffic": TRAFFIC_P2_PER_BYTE and
+                     TRAFFIC_P2_PER_BYTE * bytes_p2},
+        "roofline_pass1": {"bound": "hbm", "kernel": "row_stats_kernel (pass 1)", "achieved": ach_p1,
+                           "peak": peak, "unit": "GB/s", "frac": ach_p1 / peak,
+                           "frac_of_8TBs_nominal": ach_p1 / 8000.0, "ms_per_launch": p1,
+                           "algorithmic_bytes_per_launch": bytes_p1},
+        "roofline_step": {"achieved": ach_all, "peak": peak, "unit": "GB/s", "frac": ach_all / peak,
+                          "frac_of_8TBs_nominal": ach_all / 8000.0, "finalize_ms": fin},
+        "cpu_baseline": cpu,
+        "stats": {"n_clipped": st["n_clipped"], "mean_log_cw": st["mean_log_cw"], "loss": st["loss"]},
+    }
+    print(json.dumps(line), flush=True)
+    if dist:
+        dist.destroy_process_group()
+
+
+# DRAM traffic of pass 2 per algorithmic byte, from the ncu capture summarised under profiles/
+# (dram__bytes_read.sum + dram__bytes_write.sum of a smaller launch, which scales with rows).
+TRAFFIC_P2_PER_BYTE = None
+
+
+def run_e2e(rb, args, desc, w, logits, tok, behav, dlogits, ws, loss, token_logp, adv, stats,
+            n_tokens, dev, dist):
+    """Same step, but the inputs start in pinned HOST memory and the loss is read back to the host
+    every step.  Uses a full pinned copy of the logits when the host has room, otherwise a
+    2 GiB pinned buffer copied repeatedly into successive device slices (same bytes moved)."""
+    import psutil
+    T = logits.shape[0]
+    nbytes = logits.numel() * logits.element_size()
+    steps = max(1, min(args.e2e_steps, args.steps))
+    mode = "full pinned copy"
+    host_logits = None
+    try:
+        if psutil.virtual_memory().available > 3 * nbytes:
+            host_logits = torch.empty(logits.shape, dtype=logits.dtype, pin_memory=True)
+            host_logits.copy_(logits)
+    except Exception:
+        host_logits = None
+    if host_logits is None:
+        rows = max(1, min(T, (2 << 30) // (logits.shape[1] * logits.element_size())))
+        host_logits = torch.empty((rows, logits.shape[1]), dtype=logits.dtype, pin_memory=True)
+        host_logits.copy_(logits[:rows])
+        mode = f"{rows}-row pinned buffer reused for every slice"
+    small = {k: tok[k].pin_memory() for k in ("targets", "mask", "rewards", "group_offsets")}
+    h_behav = behav.cpu().pin_memory()
+    d = {k: torch.empty_like(v, device=dev) for k, v in small.items()}
+    d_behav = torch.empty_like(behav)
+    d_logits = torch.empty_like(logits)
+    h_loss = torch.empty(1, dtype=torch.float32).pin_memory()
+    h2d = nbytes + sum(v.numel() * v.element_size() for v in small.values()) + h_behav.numel() * 4
+    d2h = 4
+
+    def step():
+        if host_logits.shape[0] == T:
+            d_logits.copy_(host_logits, non_blocking=True)
+        else:
+            R = host_logits.shape[0]
+            for r0 in range(0, T, R):
+                n = min(R, T - r0)
+                d_logits[r0:r0 + n].copy_(host_logits[:n], non_blocking=True)
+        for k in small:
+            d[k].copy_(small[k], non_blocking=True)
+        d_behav.copy_(h_behav, non_blocking=True)
+        rb.rapid_pg_loss_fwd_bwd(desc, d_logits, d["targets"], d["mask"], d_behav, d["rewards"],
+                                 d["group_offsets"], dlogits, loss, token_logp, adv, stats, ws)
+        h_loss.copy_(loss, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        return float(h_loss[0])
+
+    step()
+    if dist:
+        dist.barrier()
+    torch.cuda.synchronize()
+    s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s.record()
+    for _ in range(steps):
+        step()
+    e.record()
+    torch.cuda.synchronize()
+    ms = s.elapsed_time(e)
+    tokens = float(n_tokens)
+    if dist:
+        t = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+        tk = torch.tensor([tokens], device=dev, dtype=torch.float64)
+        dist.all_reduce(tk, op=dist.ReduceOp.SUM)
+        tokens = float(tk.item())
+    del d_logits, host_logits
+    return {"value": tokens * steps / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+            "d2h_bytes_per_step": int(d2h), "steps": steps, "ms_per_step": ms / steps,
+            "host_buffer": mode}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--seq-len", type=int, default=0,
+                    help="shorter padded length (smaller device footprint, e.g. for profiling)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        args.warmup = max(args.warmup, 3)
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,201 @@
+/*
+ * rapid_pg.h -- C ABI of librapid_pg: the importance-weighted group-advantage policy-gradient
+ * loss of RAPID (arXiv 2510.03515) and its gradient w.r.t. the logits, as CUDA kernels for
+ * NVIDIA B200 (sm_100a).
+ *
+ * What one call computes (the two "Compute ..." lines of Algorithm 1, procedure IW-GRPG, for one
+ * mini-batch Z_h of N generations):
+ *
+ *   log pi_theta(y_t|.) = z[r, y_r] - logsumexp_v z[r, v]                  softmax policy, Sec. 3.1
+ *   s_n = sum_t m_r (log pi_theta(y_t) - log mu(y_t)),  w_n = exp(s_n)    generation-level weight,
+ *                                                                          Sec. 4.3 ("Importance-
+ *                                                                          weight clipping")
+ *   c_n = min(w_n, eta)                                                    Eq. 5 (cap; eta = 2.0
+ *                                                                          in the paper's table of
+ *                                                                          hyper-parameters)
+ *   A_n = R_n - (1/N_k) sum_{n' in group k} c_n' R_n'                      Eq. 5 (Eq. 2 when every
+ *                                                                          c is 1, Eq. 4 when
+ *                                                                          eta = +inf)
+ *   g_n = c_n A_n / N,   loss = - sum_n g_n sum_t m_r log pi_theta(y_t)    Eq. 3, with
+ *                                                                          grad pi / mu = w grad log pi
+ *                                                                          and w, A held constant
+ *   dlogits[r, v] = g_n m_r (softmax(z[r, .])_v - 1[v == y_r])            d loss / d logits
+ *
+ * Row r = n * seq_len + t of the padded token grid belongs to generation n.  `loss` is minus the
+ * paper's objective estimate (the paper takes ascent steps; this library returns the quantity
+ * to minimise), so dlogits = -(w A (onehot - softmax)) / N.
+ *
+ * Conventions, unless a parameter says otherwise:
+ *   - `desc`, `bytes` and other plain scalars are HOST memory; every array pointer is a DEVICE
+ *     pointer owned by the caller and valid on the current device.  The library allocates
+ *     nothing, keeps no state between calls and frees nothing.
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = the default stream)
+ *     and the call returns without synchronising.  Outputs are valid once the stream reaches
+ *     the end of the enqueued work.
+ *   - The return value reports what the host can see (NULL pointers, sizes, alignment, launch
+ *     errors).  Problems only the device can see never trap: a sampled token id outside
+ *     [0, vocab) makes its row count as masked and is counted in rapid_stats_t.n_bad_token; an
+ *     invalid group_offsets array sets rapid_stats_t.status, zeroes every coefficient (so
+ *     dlogits is all zero) and makes loss NaN.
+ *   - Logits must be finite.  +-inf or NaN logits give unspecified (but memory-safe) results.
+ *   - Only sm_100 devices are supported: other devices get RAPID_ERR_UNSUPPORTED.
+ */
+#ifndef RAPID_PG_H
+#define RAPID_PG_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    RAPID_OK = 0,
+    RAPID_ERR_INVALID_ARG = 1, /* NULL where an array is required, non-positive size, ld < vocab  */
+    RAPID_ERR_ALIGNMENT = 2,   /* a logits base or row pitch that is not a multiple of 16 bytes   */
+    RAPID_ERR_UNSUPPORTED = 3, /* wrong device architecture, or a size beyond a stated limit      */
+    RAPID_ERR_WORKSPACE = 4,   /* workspace NULL, misaligned (256 B) or smaller than required     */
+    RAPID_ERR_CUDA = 5,        /* a CUDA runtime call or kernel launch failed                     */
+    RAPID_ERR_TIMEOUT = 6      /* a bounded device-side wait gave up (reported in stats.status)   */
+} rapid_status_t;
+
+typedef enum { RAPID_F32 = 0, RAPID_BF16 = 1 } rapid_dtype_t;
+
+enum {
+    /* Eq. 3 exactly as printed: the outer weight is w_n, not the clipped c_n.  Default (flag
+     * clear) clips both, which is what keeps generation-level weights from blowing up.          */
+    RAPID_FLAG_OUTER_UNCLIPPED = 1u,
+    /* Normalise by the number of unmasked tokens instead of the number of generations N.        */
+    RAPID_FLAG_NORM_TOKENS = 2u,
+    /* rapid_group_advantage only: seq_log_ratio holds w_n itself, not s_n = log w_n.            */
+    RAPID_FLAG_ADV_INPUT_IS_WEIGHT = 4u,
+    /* Baseline over the other members of the group, divided by N_k - 1 (the unbiased variant
+     * shown after Eq. 4, which the paper states but does not use).                              */
+    RAPID_FLAG_LEAVE_ONE_OUT = 8u,
+    /* With LEAVE_ONE_OUT: divide by N_k, as that display is printed.                            */
+    RAPID_FLAG_LOO_LITERAL_DIVISOR = 16u
+};
+
+/* Problem descriptor (host memory, plain data, 40 bytes). */
+typedef struct rapid_desc {
+    int32_t n_seq;    /* N: generations in the mini-batch (N_step in the paper)                   */
+    int32_t seq_len;  /* L: padded response length; rows T = N * L                                */
+    int32_t vocab;    /* V                                                                        */
+    int32_t n_groups; /* K: prompts; group k is the generation range [offsets[k], offsets[k+1])  */
+    int64_t ld;       /* row pitch of logits / dlogits in ELEMENTS, >= vocab, pitch bytes % 16 == 0 */
+    int32_t dtype;    /* rapid_dtype_t of logits and dlogits                                      */
+    uint32_t flags;   /* RAPID_FLAG_* bits                                                        */
+    double eta;       /* importance-weight cap of Eq. 5; +inf gives Eq. 4; must be > 0            */
+} rapid_desc_t;
+
+/* Side statistics (DEVICE memory, written by the finalize step, 48 bytes). */
+typedef struct rapid_stats {
+    int64_t n_tokens;       /* tokens that count: mask set and target id valid                    */
+    int32_t n_clipped;      /* generations with w_n > eta (strictly)                              */
+    int32_t n_bad_token;    /* rows with mask set but target id outside [0, vocab)                */
+    int32_t n_empty_group;  /* groups with N_k = 0 (skipped)                                      */
+    int32_t status;         /* rapid_status_t seen by the device: RAPID_OK, or                    */
+                            /* RAPID_ERR_INVALID_ARG when group_offsets is not a monotone cover   */
+                            /* of [0, N)                                                          */
+    double mean_log_cw;     /* (1/N) sum_n log c_n: the staleness statistic of Sec. 4.3 / Table 3 */
+    double mean_abs_log_cw; /* (1/N) sum_n |log c_n|                                              */
+    double loss;            /* the loss in double                                                 */
+} rapid_stats_t;
+
+/* Human-readable name of a status code (static storage, never NULL). */
+const char* rapid_status_string(rapid_status_t status);
+
+/* Library version as major * 10000 + minor * 100 + patch. */
+int32_t rapid_version(void);
+
+/*
+ * Size of the scratch workspace the logits-in calls need for `desc` (16 bytes per row plus a
+ * few per generation).  `bytes` is host memory.  The workspace must be 256-byte aligned device
+ * memory; its contents need not be initialised.  Between rapid_pg_stats_chunk, rapid_pg_finalize
+ * and rapid_pg_dlogits_chunk it carries the per-row and per-generation state and must not be
+ * touched by the caller.
+ */
+rapid_status_t rapid_workspace_bytes(const rapid_desc_t* desc, size_t* bytes);
+
+/*
+ * Group advantage on its own (Eq. 2 / Eq. 4 / Eq. 5; leave-one-out by flag).
+ *   rewards        [N] float, R_n (any finite value)
+ *   seq_log_ratio  [N] double, s_n = log w_n (or w_n with RAPID_FLAG_ADV_INPUT_IS_WEIGHT);
+ *                  NULL = on-policy, every weight 1 (Eq. 2)
+ *   group_offsets  [K+1] int32, offsets[0] = 0, non-decreasing, offsets[K] = N
+ *   adv            [N] float out: the double result rounded once to float
+ *   clipped_w      [N] double out, c_n; may be NULL
+ *   stats          out, may be NULL; only status, n_clipped, n_empty_group, mean_log_cw and
+ *                  mean_abs_log_cw are meaningful here (the rest is zero)
+ * Uses desc->n_seq, n_groups, eta and flags only.  Sums run in index order in double without
+ * fused multiply-add, so the result is bit-identical to the plain definition evaluated the same
+ * way whenever the weights are identical.
+ */
+rapid_status_t rapid_group_advantage(const rapid_desc_t* desc, const float* rewards,
+                                     const double* seq_log_ratio, const int32_t* group_offsets,
+                                     float* adv, double* clipped_w, rapid_stats_t* stats,
+                                     void* stream);
+
+/*
+ * The whole path over one mini-batch whose logits are resident: two reads and one write of the
+ * logits (a first pass for the row statistics, the per-generation/per-group finalize, and one
+ * re-read pass that writes dlogits).
+ *   logits        [T, ld] of desc->dtype, row-major; only the first `vocab` entries of a row
+ *                 are used.  Base address and ld * sizeof(element) must be multiples of 16.
+ *   targets       [T] int32, the sampled token y_r
+ *   mask          [T] uint8, non-zero = the token counts; NULL = all ones.  Masked rows of
+ *                 logits are never read.
+ *   behav_logp    [T] float, log mu(y_t|.) stored by the behaviour policy at sampling time
+ *   rewards       [N] float
+ *   group_offsets [K+1] int32 (see rapid_group_advantage)
+ *   dlogits       [T, ld] out, same dtype and pitch as logits; may be the SAME buffer as logits
+ *                 (in place).  Partial overlap is not allowed.  Rows that are masked, or whose
+ *                 coefficient g_n is zero, are written as zeros.  Columns >= vocab are untouched.
+ *   loss          [1] float out
+ *   token_logp    [T] float out (0 on masked rows); may be NULL
+ *   adv           [N] float out; may be NULL
+ *   stats         out; may be NULL
+ *   workspace     rapid_workspace_bytes(desc) bytes, 256-byte aligned
+ */
+rapid_status_t rapid_pg_loss_fwd_bwd(const rapid_desc_t* desc, const void* logits,
+                                     const int32_t* targets, const uint8_t* mask,
+                                     const float* behav_logp, const float* rewards,
+                                     const int32_t* group_offsets, void* dlogits, float* loss,
+                                     float* token_logp, float* adv, rapid_stats_t* stats,
+                                     void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * The same path in three steps, for logits that are produced (or fit in memory) only a block of
+ * rows at a time.  The order is forced by the data: every generation of a group must have gone
+ * through the statistics pass before any of the group's dlogits can be written.
+ *
+ *   1. rapid_pg_stats_chunk   for every block of rows [row0, row0 + n_rows) of the [T, V] grid,
+ *                             in any order, each row exactly once
+ *   2. rapid_pg_finalize      once
+ *   3. rapid_pg_dlogits_chunk for every block again (the caller re-materialises the same logits)
+ *
+ * logits_chunk / dlogits_chunk point at row `row0` (so chunk row i is global row row0 + i) and
+ * use pitch desc->ld; targets, mask and behav_logp are the FULL [T] arrays.  The workspace is the
+ * one from rapid_workspace_bytes(desc), shared by all three steps.  dlogits_chunk may alias
+ * logits_chunk.
+ */
+rapid_status_t rapid_pg_stats_chunk(const rapid_desc_t* desc, const void* logits_chunk,
+                                    int64_t row0, int64_t n_rows, const int32_t* targets,
+                                    const uint8_t* mask, void* workspace, size_t workspace_bytes,
+                                    void* stream);
+
+rapid_status_t rapid_pg_finalize(const rapid_desc_t* desc, const float* behav_logp,
+                                 const float* rewards, const int32_t* group_offsets, float* loss,
+                                 float* token_logp, float* adv, rapid_stats_t* stats,
+                                 void* workspace, size_t workspace_bytes, void* stream);
+
+rapid_status_t rapid_pg_dlogits_chunk(const rapid_desc_t* desc, const void* logits_chunk,
+                                      void* dlogits_chunk, int64_t row0, int64_t n_rows,
+                                      const int32_t* targets, const void* workspace,
+                                      size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RAPID_PG_H */

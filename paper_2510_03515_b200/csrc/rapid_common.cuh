@@ -1,0 +1,144 @@
+// Shared device helpers and the workspace layout of librapid_pg (sm_100a only).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "rapid_pg.h"
+
+namespace rapid {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr double kLog2eD = 1.4426950408889634074;
+constexpr double kLn2D = 0.69314718055994530942;
+
+// Per-row state written by the statistics pass.
+enum : uint8_t { ROW_MASKED = 0, ROW_OK = 1, ROW_BAD_TOKEN = 2 };
+
+// Device pointers carved out of the caller's workspace.  Per row: 8 (lse) + 8 (log pi) +
+// 4 (row max) + 1 (state) bytes; per generation: a handful of doubles.
+struct Workspace {
+    double* lse;            // [T] log sum_v exp z[r, v]
+    double* token_logp;     // [T] z[r, y_r] - lse[r]
+    float* row_max;         // [T] max_v z[r, v]
+    uint8_t* row_state;     // [T] ROW_*
+    double* seq_log_ratio;  // [N] s_n
+    double* seq_logp;       // [N] S_n
+    double* weight;         // [N] w_n
+    double* clipped_w;      // [N] c_n
+    double* adv;            // [N] A_n
+    double* coef;           // [N] g_n
+    double* coef_log2;      // [N] log2 |g_n| (-inf when g_n == 0)
+    int32_t* seq_tokens;    // [N]
+    int32_t* seq_bad;       // [N] rows with a target id outside [0, V)
+    rapid_stats_t* stats;   // [1]
+};
+
+__host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Carve `base` (256-byte aligned).  Returns the number of bytes used.
+__host__ inline size_t carve_workspace(const rapid_desc_t& d, void* base, Workspace* w) {
+    const size_t T = (size_t)d.n_seq * (size_t)d.seq_len;
+    const size_t N = (size_t)d.n_seq;
+    size_t off = 0;
+    char* p = static_cast<char*>(base);
+    auto take = [&](size_t bytes) {
+        char* q = p ? p + off : nullptr;
+        off = align_up(off + bytes, 256);
+        return q;
+    };
+    Workspace ws;
+    ws.lse = reinterpret_cast<double*>(take(T * 8));
+    ws.token_logp = reinterpret_cast<double*>(take(T * 8));
+    ws.row_max = reinterpret_cast<float*>(take(T * 4));
+    ws.row_state = reinterpret_cast<uint8_t*>(take(T));
+    ws.seq_log_ratio = reinterpret_cast<double*>(take(N * 8));
+    ws.seq_logp = reinterpret_cast<double*>(take(N * 8));
+    ws.weight = reinterpret_cast<double*>(take(N * 8));
+    ws.clipped_w = reinterpret_cast<double*>(take(N * 8));
+    ws.adv = reinterpret_cast<double*>(take(N * 8));
+    ws.coef = reinterpret_cast<double*>(take(N * 8));
+    ws.coef_log2 = reinterpret_cast<double*>(take(N * 8));
+    ws.seq_tokens = reinterpret_cast<int32_t*>(take(N * 4));
+    ws.seq_bad = reinterpret_cast<int32_t*>(take(N * 4));
+    ws.stats = reinterpret_cast<rapid_stats_t*>(take(sizeof(rapid_stats_t)));
+    if (w) *w = ws;
+    return off;
+}
+
+#ifdef __CUDACC__
+
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// The two halves of a packed pair of bf16 values, widened exactly to float.
+__device__ __forceinline__ float bf16_lo(uint32_t p) { return __uint_as_float(p << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t p) { return __uint_as_float(p & 0xffff0000u); }
+
+// max of two packed bf16 pairs, element-wise
+__device__ __forceinline__ uint32_t bf16x2_max(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+
+// round two floats to a packed bf16 pair (lo in the low half), round-to-nearest-even
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+// 16-byte streaming load (read once, do not keep in L1) and store
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) { return __ldcs(p); }
+__device__ __forceinline__ void st_stream(uint4* p, uint4 v) { __stcs(p, v); }
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ long long warp_sum(long long v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ int warp_sum(int v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+#endif  // __CUDACC__
+
+// Host-side launchers (each enqueues on `stream` and returns the launch status).
+cudaError_t launch_row_stats(const rapid_desc_t& d, const void* logits_chunk, int64_t row0,
+                             int64_t n_rows, const int32_t* targets, const uint8_t* mask,
+                             const Workspace& ws, int sm_count, cudaStream_t stream);
+cudaError_t launch_seq_reduce(const rapid_desc_t& d, const float* behav_logp, float* token_logp_out,
+                              const Workspace& ws, cudaStream_t stream);
+cudaError_t launch_finalize(const rapid_desc_t& d, const float* rewards,
+                            const int32_t* group_offsets, float* loss, float* adv,
+                            rapid_stats_t* stats_out, const Workspace& ws, cudaStream_t stream);
+cudaError_t launch_group_advantage(const rapid_desc_t& d, const float* rewards,
+                                   const double* seq_log_ratio, const int32_t* group_offsets,
+                                   float* adv, double* clipped_w, rapid_stats_t* stats_out,
+                                   cudaStream_t stream);
+cudaError_t launch_dlogits(const rapid_desc_t& d, const void* logits_chunk, void* dlogits_chunk,
+                           int64_t row0, int64_t n_rows, const int32_t* targets,
+                           const Workspace& ws, int sm_count, cudaStream_t stream);
+
+}  // namespace rapid

@@ -1,0 +1,246 @@
+// Pass 1: per-row log-sum-exp over the vocabulary and the sampled token's log-probability
+// (the softmax policy's log pi_theta(y_t|.), the quantity that Eq. 3 and Eq. 5 are built from).
+//
+// One CTA streams one row at a time with 128-bit loads; rows are taken grid-stride.  Masked rows
+// and rows with an invalid token id are not read.
+//
+// bf16 logits: one sweep, online max/sum per thread in float (base-2 exponentials on the MUFU
+// pipe), combined across the CTA in double.
+// fp32 logits: the tolerance on the loss is tight (a generation sums thousands of token
+// log-probs), so the row maximum is found first and the exponentials are then summed against
+// that exact maximum, four at a time in float and accumulated in double.  The second sweep of a
+// row hits L2.
+#include "rapid_common.cuh"
+
+namespace rapid {
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+
+// ---- bf16 ------------------------------------------------------------------------------------
+
+template <int U>
+__device__ __forceinline__ void bf16_batch(const uint4 (&q)[U], float& m, float& s0, float& s1) {
+    uint32_t mx = bf16x2_max(bf16x2_max(q[0].x, q[0].y), bf16x2_max(q[0].z, q[0].w));
+#pragma unroll
+    for (int j = 1; j < U; ++j)
+        mx = bf16x2_max(mx, bf16x2_max(bf16x2_max(q[j].x, q[j].y), bf16x2_max(q[j].z, q[j].w)));
+    const float bm = fmaxf(bf16_lo(mx), bf16_hi(mx));
+    if (bm > m) {  // rare after the first few batches
+        const float f = ex2_approx((m - bm) * kLog2e);
+        s0 *= f;
+        s1 *= f;
+        m = bm;
+    }
+    const float nm = -m * kLog2e;
+#pragma unroll
+    for (int j = 0; j < U; ++j) {
+        const uint32_t w[4] = {q[j].x, q[j].y, q[j].z, q[j].w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            s0 += ex2_approx(fmaf(bf16_lo(w[k]), kLog2e, nm));
+            s1 += ex2_approx(fmaf(bf16_hi(w[k]), kLog2e, nm));
+        }
+    }
+}
+
+__device__ __forceinline__ void row_sweep_bf16(const uint16_t* row, int vocab, float& m_out,
+                                               float& s_out) {
+    constexpr int U = 4;
+    const int tid = threadIdx.x;
+    const int nvec = vocab >> 3;
+    const uint4* rv = reinterpret_cast<const uint4*>(row);
+    float m = -INFINITY, s0 = 0.f, s1 = 0.f;
+    int v = tid;
+    for (; v + (U - 1) * kThreads < nvec; v += U * kThreads) {
+        uint4 q[U];
+#pragma unroll
+        for (int j = 0; j < U; ++j) q[j] = ld_stream(rv + v + j * kThreads);
+        bf16_batch<U>(q, m, s0, s1);
+    }
+    for (; v < nvec; v += kThreads) {
+        uint4 q[1];
+        q[0] = ld_stream(rv + v);
+        bf16_batch<1>(q, m, s0, s1);
+    }
+    // ragged tail (vocab not a multiple of 8): one element per thread
+    const int e = (nvec << 3) + tid;
+    if (e < vocab) {
+        const float z = __uint_as_float(((uint32_t)row[e]) << 16);
+        if (z > m) {
+            const float f = ex2_approx((m - z) * kLog2e);
+            s0 *= f;
+            s1 *= f;
+            m = z;
+        }
+        s0 += ex2_approx((z - m) * kLog2e);
+    }
+    m_out = m;
+    s_out = s0 + s1;
+}
+
+// ---- fp32 ------------------------------------------------------------------------------------
+
+__device__ __forceinline__ float row_max_f32(const float* row, int vocab) {
+    constexpr int U = 4;
+    const int tid = threadIdx.x;
+    const int nvec = vocab >> 2;
+    const float4* rv = reinterpret_cast<const float4*>(row);
+    float m = -INFINITY;
+    int v = tid;
+    for (; v + (U - 1) * kThreads < nvec; v += U * kThreads) {
+        float4 q[U];
+#pragma unroll
+        for (int j = 0; j < U; ++j) q[j] = __ldg(rv + v + j * kThreads);
+#pragma unroll
+        for (int j = 0; j < U; ++j) m = fmaxf(m, fmaxf(fmaxf(q[j].x, q[j].y), fmaxf(q[j].z, q[j].w)));
+    }
+    for (; v < nvec; v += kThreads) {
+        const float4 q = __ldg(rv + v);
+        m = fmaxf(m, fmaxf(fmaxf(q.x, q.y), fmaxf(q.z, q.w)));
+    }
+    const int e = (nvec << 2) + tid;
+    if (e < vocab) m = fmaxf(m, __ldg(row + e));
+    return m;
+}
+
+__device__ __forceinline__ double row_expsum_f32(const float* row, int vocab, float M) {
+    constexpr int U = 4;
+    const int tid = threadIdx.x;
+    const int nvec = vocab >> 2;
+    const float4* rv = reinterpret_cast<const float4*>(row);
+    double acc = 0.0;
+    int v = tid;
+    for (; v + (U - 1) * kThreads < nvec; v += U * kThreads) {
+        float4 q[U];
+#pragma unroll
+        for (int j = 0; j < U; ++j) q[j] = __ldcs(rv + v + j * kThreads);
+#pragma unroll
+        for (int j = 0; j < U; ++j)
+            acc += (double)((expf(q[j].x - M) + expf(q[j].y - M)) +
+                            (expf(q[j].z - M) + expf(q[j].w - M)));
+    }
+    for (; v < nvec; v += kThreads) {
+        const float4 q = __ldcs(rv + v);
+        acc += (double)((expf(q.x - M) + expf(q.y - M)) + (expf(q.z - M) + expf(q.w - M)));
+    }
+    const int e = (nvec << 2) + tid;
+    if (e < vocab) acc += (double)expf(__ldg(row + e) - M);
+    return acc;
+}
+
+// ---- kernel ----------------------------------------------------------------------------------
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads)
+row_stats_kernel(const void* __restrict__ logits, int64_t ld, int vocab, int64_t row0,
+                 int64_t n_rows, const int32_t* __restrict__ targets,
+                 const uint8_t* __restrict__ mask, Workspace ws) {
+    __shared__ float sh_m[kWarps];
+    __shared__ double sh_s[kWarps];
+    __shared__ float sh_bcast;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    for (int64_t i = blockIdx.x; i < n_rows; i += gridDim.x) {
+        const int64_t r = row0 + i;
+        const bool on = mask ? (mask[r] != 0) : true;
+        const int32_t y = targets[r];
+        if (!on || y < 0 || y >= vocab) {  // uniform across the CTA
+            if (tid == 0) {
+                ws.row_state[r] = on ? ROW_BAD_TOKEN : ROW_MASKED;
+                ws.lse[r] = 0.0;
+                ws.token_logp[r] = 0.0;
+                ws.row_max[r] = 0.f;
+            }
+            continue;
+        }
+
+        float M;
+        double S;  // sum_v exp(z_v - M) for this thread's share, then the row
+        double zy;
+        if (DT == RAPID_BF16) {
+            const uint16_t* row = static_cast<const uint16_t*>(logits) + i * ld;
+            float m, s;
+            row_sweep_bf16(row, vocab, m, s);
+            const float wm = warp_max(m);
+            // a thread (or a whole warp, for a tiny vocabulary) that saw nothing has m = -inf, s = 0
+            s *= (m == wm) ? 1.f : ex2_approx((m - wm) * kLog2e);
+            s = warp_sum(s);
+            if (lane == 0) {
+                sh_m[warp] = wm;
+                sh_s[warp] = (double)s;
+            }
+            __syncthreads();
+            if (tid == 0) {
+                float mm = sh_m[0];
+                for (int w = 1; w < kWarps; ++w) mm = fmaxf(mm, sh_m[w]);
+                double tot = 0.0;
+                for (int w = 0; w < kWarps; ++w)
+                    tot += sh_s[w] * (double)ex2_approx((sh_m[w] - mm) * kLog2e);
+                M = mm;
+                S = tot;
+                zy = (double)__uint_as_float(((uint32_t)row[y]) << 16);
+            }
+        } else {
+            const float* row = static_cast<const float*>(logits) + i * ld;
+            float m = warp_max(row_max_f32(row, vocab));
+            if (lane == 0) sh_m[warp] = m;
+            __syncthreads();
+            if (tid == 0) {
+                float mm = sh_m[0];
+                for (int w = 1; w < kWarps; ++w) mm = fmaxf(mm, sh_m[w]);
+                sh_bcast = mm;
+            }
+            __syncthreads();
+            M = sh_bcast;
+            double s = warp_sum(row_expsum_f32(row, vocab, M));
+            if (lane == 0) sh_s[warp] = s;
+            __syncthreads();
+            if (tid == 0) {
+                double tot = 0.0;
+                for (int w = 0; w < kWarps; ++w) tot += sh_s[w];
+                S = tot;
+                zy = (double)row[y];
+            }
+        }
+        if (tid == 0) {
+            const double lse = (double)M + log(S);
+            ws.lse[r] = lse;
+            ws.token_logp[r] = zy - lse;
+            ws.row_max[r] = M;
+            ws.row_state[r] = ROW_OK;
+        }
+        __syncthreads();  // shared scratch is reused by the next row
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_row_stats(const rapid_desc_t& d, const void* logits_chunk, int64_t row0,
+                             int64_t n_rows, const int32_t* targets, const uint8_t* mask,
+                             const Workspace& ws, int sm_count, cudaStream_t stream) {
+    if (n_rows <= 0) return cudaSuccess;
+    int per_sm = 0;
+    cudaError_t e;
+    if (d.dtype == RAPID_BF16)
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, row_stats_kernel<RAPID_BF16>,
+                                                          kThreads, 0);
+    else
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, row_stats_kernel<RAPID_F32>,
+                                                          kThreads, 0);
+    if (e != cudaSuccess) return e;
+    if (per_sm < 1) per_sm = 1;
+    int64_t grid = (int64_t)sm_count * per_sm;
+    if (grid > n_rows) grid = n_rows;
+    if (d.dtype == RAPID_BF16)
+        row_stats_kernel<RAPID_BF16><<<(unsigned)grid, kThreads, 0, stream>>>(
+            logits_chunk, d.ld, d.vocab, row0, n_rows, targets, mask, ws);
+    else
+        row_stats_kernel<RAPID_F32><<<(unsigned)grid, kThreads, 0, stream>>>(
+            logits_chunk, d.ld, d.vocab, row0, n_rows, targets, mask, ws);
+    return cudaGetLastError();
+}
+
+}  // namespace rapid

@@ -1,0 +1,228 @@
+"""GPU parity: the CUDA library (through its C ABI) against the float64 CPU oracle on the same
+seeded inputs, element by element, at sizes the oracle finishes in seconds."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+import oracle  # noqa: E402
+from paper_2510_03515_b200 import binding as rb  # noqa: E402
+from paper_2510_03515_b200 import synth  # noqa: E402
+from parity_util import compare, run_both  # noqa: E402
+
+
+def _dt(w):
+    return synth.torch_dtype(w)
+
+
+def test_config_tiny_full_size():
+    """4 prompts x 8 samples, 64 tokens, V = 4096, fp32, seed 0: every element compared."""
+    w = synth.CONFIGS["tiny"]
+    b = synth.make_batch(w)
+    o, g = run_both(b, w.n_seq, w.seq_len)
+    r = compare(o, g, _dt(w), w.seq_len)
+    assert np.abs(g["dlogits"].sum(1)).max() < 1e-6
+
+
+@pytest.mark.parametrize("in_place", [False, True])
+def test_config_slm_scaled(in_place):
+    """SLM mini-batch shape at full vocabulary (151936, bf16, boosted sampled logit, ragged
+    lengths with trailing padding), fewer and shorter generations so the oracle takes seconds."""
+    w = synth.CONFIGS["slm"].scaled(n_prompts=2, group_size=4, seq_len=40, len_lo=10)
+    b = synth.make_batch(w)
+    o, g = run_both(b, w.n_seq, w.seq_len, in_place=in_place)
+    compare(o, g, _dt(w), w.seq_len)
+    assert (b["mask"] == 0).any()
+
+
+@pytest.mark.parametrize("sigma", synth.STALE_SIGMAS)
+def test_config_stale_scaled(sigma):
+    """Staleness sweep: sigma in {0, .1, .5, 1, 2}; includes an all-zero and an all-one group."""
+    w = synth.CONFIGS["stale"].scaled(n_prompts=4, group_size=4, seq_len=24, behav_sigma=sigma)
+    b = synth.make_batch(w)
+    o, g = run_both(b, w.n_seq, w.seq_len)
+    compare(o, g, _dt(w), w.seq_len)
+    assert np.all(o["adv64"][:4] == 0.0)  # all-zero rewards: no std division, exactly zero
+    if sigma >= 1:
+        assert o["n_clipped"] > 0
+
+
+def test_config_long_scaled_chunked():
+    """Long sequences, V = 32000 fp32, 30% trailing padding, through the chunked three-step API
+    with a ragged last chunk; also equals the one-call form."""
+    w = synth.CONFIGS["long"].scaled(n_prompts=2, group_size=4, seq_len=640)
+    b = synth.make_batch(w)
+    o, g = run_both(b, w.n_seq, w.seq_len)
+    compare(o, g, _dt(w), w.seq_len)
+
+    dev = torch.device("cuda")
+    T, V = b["logits"].shape
+    behav = torch.from_numpy(o["token_logp"]).double().add(b["behav_noise"].double()).float().to(dev)
+    desc = rb.make_desc(w.n_seq, w.seq_len, V, w.n_prompts, torch.float32)
+    ws = rb.alloc_workspace(desc, dev)
+    tg, mk = b["targets"].to(dev), b["mask"].to(dev)
+    chunk = 1500
+    starts = list(range(0, T, chunk))
+    for r0 in reversed(starts):  # any order
+        n = min(chunk, T - r0)
+        rb.rapid_pg_stats_chunk(desc, b["logits"][r0:r0 + n].to(dev), r0, n, tg, mk, ws)
+    loss = torch.zeros(1, device=dev)
+    tl = torch.zeros(T, device=dev)
+    adv = torch.zeros(w.n_seq, device=dev)
+    st = rb.alloc_stats(dev)
+    rb.rapid_pg_finalize(desc, behav, b["rewards"].to(dev), b["group_offsets"].to(dev), loss, tl, adv, st, ws)
+    dz = torch.empty((T, V), device=dev)
+    for r0 in starts:
+        n = min(chunk, T - r0)
+        zc = b["logits"][r0:r0 + n].to(dev)
+        rb.rapid_pg_dlogits_chunk(desc, zc, dz[r0:r0 + n], r0, n, tg, ws)
+    torch.cuda.synchronize()
+    g2 = {"loss": loss.item(), "token_logp": tl.cpu().numpy(), "adv": adv.cpu().numpy(),
+          "stats": rb.read_stats(st), "dlogits": dz.cpu().numpy()}
+    compare(o, g2, torch.float32, w.seq_len)
+    # the chunked form and the one-call form run the same kernels on the same rows
+    assert g2["loss"] == g["loss"]
+    np.testing.assert_array_equal(g2["dlogits"], g["dlogits"])
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("V,pad", [(1, 7), (2, 6), (7, 1), (8, 0), (9, 7), (255, 1), (257, 7),
+                                   (1000, 0), (4099, 5), (33000, 0)])
+def test_ragged_vocab_and_row_pitch(dtype, V, pad):
+    """Vocabulary sizes around the vector width and the per-thread batch, with a padded pitch."""
+    per = 4 if dtype == "f32" else 8
+    pad = (-V) % per + (per if pad else 0)  # pitch must be a multiple of 16 bytes
+    w = synth.Workload("edge", 2, 3, 5, V, dtype, 2.0, 3.0 if V > 1 else 0.0, "uniform", len_lo=0,
+                       behav_sigma=0.3, reward_mode="per_prompt", seed=100 + V)
+    b = synth.make_batch(w)
+    o, g = run_both(b, w.n_seq, w.seq_len, ld_pad=pad)
+    compare(o, g, _dt(w), w.seq_len)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("flags", [0, rb.FLAG_OUTER_UNCLIPPED, rb.FLAG_NORM_TOKENS,
+                                   rb.FLAG_LEAVE_ONE_OUT, rb.FLAG_LEAVE_ONE_OUT | rb.FLAG_LOO_LITERAL_DIVISOR,
+                                   rb.FLAG_OUTER_UNCLIPPED | rb.FLAG_NORM_TOKENS])
+@pytest.mark.parametrize("eta", [2.0, math.inf, 0.5])
+def test_flags_and_eta(dtype, flags, eta):
+    w = synth.Workload("flags", 3, 4, 9, 515, dtype, 2.0, 4.0, "uniform", len_lo=1,
+                       behav_sigma=0.25, reward_mode="per_prompt", seed=7)
+    b = synth.make_batch(w)
+    b["rewards"] = torch.randn(w.n_seq, generator=torch.Generator().manual_seed(3))  # real-valued rewards
+    o, g = run_both(b, w.n_seq, w.seq_len, eta=eta, flags=flags)
+    compare(o, g, _dt(w), w.seq_len)
+
+
+def test_degenerate_shapes():
+    """L = 1; groups of one; an empty group; a generation with no unmasked token; bad token ids."""
+    V = 300
+    N, L = 6, 1
+    gen = torch.Generator().manual_seed(11)
+    b = {
+        "logits": torch.randn((N * L, V), generator=gen) * 2,
+        "targets": torch.randint(0, V, (N * L,), generator=gen, dtype=torch.int64).to(torch.int32),
+        "mask": torch.tensor([1, 1, 0, 1, 1, 1], dtype=torch.uint8),
+        "rewards": torch.tensor([1.0, 0.0, 1.0, 1.0, 0.5, -2.0]),
+        "group_offsets": torch.tensor([0, 1, 1, 3, 6], dtype=torch.int32),  # sizes 1, 0, 2, 3
+        "behav_noise": torch.randn(N * L, generator=gen) * 0.5,
+    }
+    b["targets"][4] = V        # out of range: row counts as masked, is reported
+    b["targets"][5] = -1
+    o, g = run_both(b, N, L)
+    compare(o, g, torch.float32, L)
+    assert g["stats"]["n_bad_token"] == 2 and g["stats"]["n_empty_group"] == 1
+    assert g["stats"]["n_tokens"] == 3
+
+
+def test_everything_masked():
+    w = synth.Workload("allmasked", 2, 2, 4, 64, "bf16", 1.0, 0.0, "full", seed=5)
+    b = synth.make_batch(w)
+    b["mask"] = torch.zeros_like(b["mask"])
+    o, g = run_both(b, w.n_seq, w.seq_len)
+    assert g["loss"] == 0.0 and np.all(g["dlogits"] == 0.0) and g["stats"]["n_tokens"] == 0
+    compare(o, g, torch.bfloat16, w.seq_len)
+    o, g = run_both(b, w.n_seq, w.seq_len, flags=rb.FLAG_NORM_TOKENS)  # Z = 0 tokens: still finite
+    assert g["loss"] == 0.0 and np.all(g["dlogits"] == 0.0)
+
+
+def test_mask_null_means_all_ones():
+    w = synth.Workload("nomask", 2, 2, 6, 1024, "f32", 2.0, 0.0, "full", seed=6)
+    b = synth.make_batch(w)
+    del b["mask"]
+    o, g = run_both(b, w.n_seq, w.seq_len)
+    compare(o, g, torch.float32, w.seq_len)
+    assert g["stats"]["n_tokens"] == w.n_rows
+
+
+def test_invalid_group_offsets_reported_by_device():
+    w = synth.Workload("badgroups", 2, 2, 3, 128, "f32", 1.0, 0.0, "full", seed=8)
+    b = synth.make_batch(w)
+    dev = torch.device("cuda")
+    for bad in ([0, 3, 2, 4], [1, 2, 4], [0, 2, 5]):
+        go = torch.tensor(bad, dtype=torch.int32, device=dev)
+        z = b["logits"].to(dev)
+        res = rb.pg_loss(z, b["targets"].to(dev), b["mask"].to(dev), torch.zeros(w.n_rows, device=dev),
+                         b["rewards"].to(dev), go, w.n_seq, w.seq_len)
+        torch.cuda.synchronize()
+        st = rb.read_stats(res.stats)
+        assert st["status"] == rb.RAPID_ERR_INVALID_ARG
+        assert math.isnan(res.loss.item())
+        assert torch.all(res.dlogits == 0)
+
+
+# ---- rapid_group_advantage on its own: bit-exact ----------------------------------------------------
+
+def _adv_gpu(R, slr, go, eta, flags):
+    dev = torch.device("cuda")
+    N, K = len(R), len(go) - 1
+    desc = rb.RapidDesc(N, 1, 1, K, 1, rb.RAPID_F32, flags, eta)
+    adv = torch.full((N,), float("nan"), device=dev)
+    cw = torch.full((N,), float("nan"), dtype=torch.float64, device=dev)
+    st = rb.alloc_stats(dev)
+    rb.rapid_group_advantage(desc, torch.from_numpy(R).to(dev),
+                             None if slr is None else torch.from_numpy(slr).to(dev),
+                             torch.from_numpy(go).to(dev), adv, cw, st)
+    torch.cuda.synchronize()
+    return adv.cpu().numpy(), cw.cpu().numpy(), rb.read_stats(st)
+
+
+@pytest.mark.parametrize("flags", [0, rb.FLAG_LEAVE_ONE_OUT, rb.FLAG_LEAVE_ONE_OUT | rb.FLAG_LOO_LITERAL_DIVISOR])
+@pytest.mark.parametrize("eta", [2.0, math.inf])
+def test_group_advantage_bit_exact(flags, eta):
+    rng = np.random.default_rng(17)
+    sizes = [8] * 16 + [1, 3, 16, 5, 2, 7] + [4] * 300
+    go = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int32)
+    N = int(go[-1])
+    for R in ((rng.random(N) < 0.4).astype(np.float32), rng.normal(0, 1, N).astype(np.float32)):
+        s = rng.normal(0, 1.0, N)
+        # (a) identical weights on both sides: bit-exact by construction
+        w = np.exp(s)
+        ref = oracle.group_advantage(R, w, go, eta, flags | oracle.FLAG_ADV_INPUT_IS_WEIGHT)
+        adv, cw, st = _adv_gpu(R, w, go, eta, flags | rb.FLAG_ADV_INPUT_IS_WEIGHT)
+        assert np.array_equal(adv.view(np.uint32), ref["adv32"].view(np.uint32))
+        assert np.array_equal(cw, ref["clipped_w"])
+        assert st["n_clipped"] == int((w > eta).sum()) and st["status"] == 0
+        assert st["mean_log_cw"] == pytest.approx(np.log(np.minimum(w, eta)).mean(), abs=1e-12)
+        # (b) log-ratios in: exp() may differ in the last double bit between the two libraries;
+        #     any float32 difference is then at most one ulp
+        ref = oracle.group_advantage(R, s, go, eta, flags)
+        adv, cw, st = _adv_gpu(R, s, go, eta, flags)
+        ulp = np.abs(adv.view(np.int32).astype(np.int64) - ref["adv32"].view(np.int32).astype(np.int64))
+        assert ulp.max() <= 1
+        # (c) on-policy (Eq. 2): no weights at all, exact
+        ref = oracle.group_advantage(R, None, go, eta, flags)
+        adv, cw, st = _adv_gpu(R, None, go, eta, flags)
+        assert np.array_equal(adv.view(np.uint32), ref["adv32"].view(np.uint32))
+        assert st["n_clipped"] == 0 and st["mean_log_cw"] == 0.0
+
+
+def test_group_advantage_zero_sum_on_device():
+    """Eq. 2 advantages sum to zero within each group (checked on the device's own output)."""
+    rng = np.random.default_rng(19)
+    go = (np.arange(65) * 8).astype(np.int32)
+    R = (rng.random(512) < 0.3).astype(np.float32)
+    adv, _, _ = _adv_gpu(R, None, go, 2.0, 0)
+    assert np.abs(adv.reshape(64, 8).astype(np.float64).sum(1)).max() < 1e-6
