@@ -71,7 +71,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.gpu_id}", f"--query-gpu={self.FIELDS}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "50"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
@@ -302,7 +302,7 @@ def run_ours(args):
 
     # ---- end to end through the public call with HOST buffers ------------------------------------
     e2e = None
-    if rank == 0 or dist:
+    if not args.skip_e2e:
         e2e = run_e2e(rb, args, desc, w, logits, tok, behav, dlogits, ws, loss, token_logp, adv, stats,
                       n_tokens, dev, dist)
 
@@ -310,9 +310,11 @@ def run_ours(args):
         if dist:
             dist.destroy_process_group()
         return
-    cpu = oracle_sample(w, target_seconds=10.0) if world == 1 or rank == 0 else None
-    for k in ("seconds", "tokens"):
-        cpu.pop(k, None)
+    cpu = None
+    if not args.skip_cpu:
+        cpu = oracle_sample(w, target_seconds=10.0)
+        for k in ("seconds", "tokens"):
+            cpu.pop(k, None)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
@@ -425,10 +427,12 @@ def run_e2e(rb, args, desc, w, logits, tok, behav, dlogits, ws, loss, token_logp
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--skip-e2e", action="store_true", help="leave out the host-buffer leg (profiling)")
+    ap.add_argument("--skip-cpu", action="store_true", help="leave out the CPU oracle timing (profiling)")
     ap.add_argument("--seq-len", type=int, default=0,
                     help="shorter padded length (smaller device footprint, e.g. for profiling)")
     args = ap.parse_args()

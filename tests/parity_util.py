@@ -39,6 +39,9 @@ def run_both(batch, n_seq, seq_len, eta=2.0, flags=0, in_place=False, want_dlogi
     """Returns (oracle dict, gpu dict of numpy arrays).  `batch` holds CPU tensors."""
     logits = batch["logits"]
     T, V = logits.shape
+    per = 16 // logits.element_size()
+    if (V + ld_pad) % per:  # the row pitch must be a multiple of 16 bytes
+        ld_pad += (-(V + ld_pad)) % per
     if ld_pad:
         padded = torch.full((T, V + ld_pad), 77.0, dtype=logits.dtype)
         padded[:, :V] = logits
