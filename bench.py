@@ -242,7 +242,7 @@ def run_ours(args):
         rb.rapid_pg_finalize(desc, behav, rewards, go, loss, token_logp, adv, stats, ws)
         if ev:
             ev[2].record()
-        rb.rapid_pg_dlogits_chunk(desc, logits, dlogits, 0, T, targets, ws)
+        rb.rapid_pg_dlogits_chunk(desc, logits, dlogits, 0, T, targets, stats, ws)
         if ev:
             ev[3].record()
 

@@ -179,6 +179,12 @@ rapid_status_t rapid_pg_loss_fwd_bwd(const rapid_desc_t* desc, const void* logit
  * use pitch desc->ld; targets, mask and behav_logp are the FULL [T] arrays.  The workspace is the
  * one from rapid_workspace_bytes(desc), shared by all three steps.  dlogits_chunk may alias
  * logits_chunk.
+ *
+ * The kernels move data with asynchronous bulk copies and wait for them on barriers; every such
+ * wait is bounded (a few seconds).  A wait that gives up never traps: in the statistics pass the
+ * row is marked and rapid_pg_finalize reports RAPID_ERR_TIMEOUT in stats->status with a NaN loss;
+ * in the dlogits pass the status word of `stats` (optional; pass the struct that finalize wrote)
+ * is raised to RAPID_ERR_TIMEOUT and the affected rows of dlogits are unspecified.
  */
 rapid_status_t rapid_pg_stats_chunk(const rapid_desc_t* desc, const void* logits_chunk,
                                     int64_t row0, int64_t n_rows, const int32_t* targets,
@@ -192,8 +198,8 @@ rapid_status_t rapid_pg_finalize(const rapid_desc_t* desc, const float* behav_lo
 
 rapid_status_t rapid_pg_dlogits_chunk(const rapid_desc_t* desc, const void* logits_chunk,
                                       void* dlogits_chunk, int64_t row0, int64_t n_rows,
-                                      const int32_t* targets, const void* workspace,
-                                      size_t workspace_bytes, void* stream);
+                                      const int32_t* targets, rapid_stats_t* stats,
+                                      void* workspace, size_t workspace_bytes, void* stream);
 
 #ifdef __cplusplus
 }

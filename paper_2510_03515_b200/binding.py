@@ -90,7 +90,7 @@ def lib():
         L.rapid_pg_finalize.restype = C.c_int
         L.rapid_pg_finalize.argtypes = [dp] + [vp] * 8 + [sz, vp]
         L.rapid_pg_dlogits_chunk.restype = C.c_int
-        L.rapid_pg_dlogits_chunk.argtypes = [dp, vp, vp, i64, i64, vp, vp, sz, vp]
+        L.rapid_pg_dlogits_chunk.argtypes = [dp, vp, vp, i64, i64, vp, vp, vp, sz, vp]
         _lib = L
     return _lib
 
@@ -191,9 +191,10 @@ def rapid_pg_finalize(desc: RapidDesc, behav_logp: torch.Tensor, rewards: torch.
 
 def rapid_pg_dlogits_chunk(desc: RapidDesc, logits_chunk: torch.Tensor,
                            dlogits_chunk: torch.Tensor, row0: int, n_rows: int,
-                           targets: torch.Tensor, workspace: torch.Tensor) -> None:
+                           targets: torch.Tensor, stats: Optional[torch.Tensor],
+                           workspace: torch.Tensor) -> None:
     _check(lib().rapid_pg_dlogits_chunk(C.byref(desc), _ptr(logits_chunk), _ptr(dlogits_chunk),
-                                        row0, n_rows, _ptr(targets), _ptr(workspace),
+                                        row0, n_rows, _ptr(targets), _ptr(stats), _ptr(workspace),
                                         workspace.numel(), _stream()), "rapid_pg_dlogits_chunk")
 
 

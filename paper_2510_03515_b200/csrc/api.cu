@@ -131,8 +131,8 @@ rapid_status_t rapid_pg_finalize(const rapid_desc_t* desc, const float* behav_lo
 
 rapid_status_t rapid_pg_dlogits_chunk(const rapid_desc_t* desc, const void* logits_chunk,
                                       void* dlogits_chunk, int64_t row0, int64_t n_rows,
-                                      const int32_t* targets, const void* workspace,
-                                      size_t workspace_bytes, void* stream) {
+                                      const int32_t* targets, rapid_stats_t* stats,
+                                      void* workspace, size_t workspace_bytes, void* stream) {
     rapid_status_t s = check_desc_full(desc);
     if (s != RAPID_OK) return s;
     const int64_t T = (int64_t)desc->n_seq * desc->seq_len;
@@ -149,8 +149,8 @@ rapid_status_t rapid_pg_dlogits_chunk(const rapid_desc_t* desc, const void* logi
     if ((s = check_workspace(desc, workspace, workspace_bytes, &ws)) != RAPID_OK) return s;
     int sms = 0;
     if ((s = check_device(&sms)) != RAPID_OK) return s;
-    return cuda_status(launch_dlogits(*desc, logits_chunk, dlogits_chunk, row0, n_rows, targets, ws,
-                                      sms, static_cast<cudaStream_t>(stream)));
+    return cuda_status(launch_dlogits(*desc, logits_chunk, dlogits_chunk, row0, n_rows, targets, stats,
+                                      ws, sms, static_cast<cudaStream_t>(stream)));
 }
 
 rapid_status_t rapid_pg_loss_fwd_bwd(const rapid_desc_t* desc, const void* logits,
@@ -179,8 +179,8 @@ rapid_status_t rapid_pg_loss_fwd_bwd(const rapid_desc_t* desc, const void* logit
     s = rapid_pg_finalize(desc, behav_logp, rewards, group_offsets, loss, token_logp, adv, stats,
                           workspace, workspace_bytes, stream);
     if (s != RAPID_OK) return s;
-    return rapid_pg_dlogits_chunk(desc, logits, dlogits, 0, T, targets, workspace, workspace_bytes,
-                                  stream);
+    return rapid_pg_dlogits_chunk(desc, logits, dlogits, 0, T, targets, stats, workspace,
+                                  workspace_bytes, stream);
 }
 
 }  // extern "C"

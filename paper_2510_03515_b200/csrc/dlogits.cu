@@ -1,203 +1,337 @@
 // Pass 2: re-read the logits once and write
 //     dlogits[r, v] = g_n m_r (softmax(z[r, .])_v - 1[v == y_r]),
-// the derivative of the Eq. 3 surrogate loss through the log-softmax.  Rows that are masked or
-// whose coefficient g_n is zero are written as zeros without reading the logits.  Each thread
-// reads a 16-byte vector and writes the same 16 bytes, so dlogits may be the logits buffer.
+// the derivative of the Eq. 3 surrogate loss through the log-softmax.
+//
+// Two kernels, both HBM-bound:
+//
+//  zero_rows_kernel   rows that are masked, or whose coefficient g_n is zero, get zeros.  Nothing is
+//                     read: one thread per CTA issues bulk shared->global copies from a zeroed
+//                     buffer, which keeps the write stream in large bursts.
+//
+//  dlogits_kernel     live rows.  Persistent CTAs take rows grid-stride.  One producer thread
+//                     streams each row into a ring of shared-memory stages with bulk global->shared
+//                     copies, running ahead across row boundaries.  Eight consumer warps wait on a
+//                     stage's barrier, turn the logits into dlogits IN PLACE in shared memory, and
+//                     one of them sends the stage back out with a bulk shared->global copy; the
+//                     stage returns to the producer once that copy has finished reading it.  Bytes
+//                     in flight are set by the ring, not by registers, and both directions move in
+//                     bursts of kChunk bytes.  A chunk is fully read before any of it is
+//                     overwritten, so dlogits may be the logits buffer itself.
 //
 // bf16: g_n is folded into the exponent, dz = sign(g) 2^(z log2(e) - lse log2(e) + log2|g|), so the
 // inner loop is one fused multiply-add and one MUFU exponential per element.
 // fp32: p = exp((z - M) - (lse - M)) with the accurate exponential, then times g.
 #include "rapid_common.cuh"
+#include "tma_pipe.cuh"
+
+#ifndef RAPID_P2_CHUNK
+#define RAPID_P2_CHUNK 16384
+#endif
+#ifndef RAPID_P2_STAGES
+#define RAPID_P2_STAGES 6
+#endif
 
 namespace rapid {
 
 namespace {
 
-constexpr int kThreads = 256;
+constexpr int kConsumers = 256;
+constexpr int kConsumerWarps = kConsumers / 32;
+constexpr int kThreads = kConsumers + 32;  // + one producer warp
+constexpr int kChunk = RAPID_P2_CHUNK;     // bytes per stage
+constexpr int kStages = RAPID_P2_STAGES;
+constexpr int kStoreDepth = kStages - 2;   // bulk stores allowed to be reading their stage
+constexpr int kVecPerChunk = kChunk / 16;
+constexpr int kVecPerThread = kVecPerChunk / kConsumers;
+static_assert(kVecPerChunk % kConsumers == 0, "chunk must be a multiple of 16 B x consumers");
+static_assert(kStages >= 3, "need a stage to load, one to work on and one to store");
 
-template <int U>
-__device__ __forceinline__ void dz_batch_bf16(uint4 (&q)[U], float c, uint32_t sign2) {
-#pragma unroll
-    for (int j = 0; j < U; ++j) {
-        uint32_t w[4] = {q[j].x, q[j].y, q[j].z, q[j].w};
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const float lo = ex2_approx(fmaf(bf16_lo(w[k]), kLog2e, c));
-            const float hi = ex2_approx(fmaf(bf16_hi(w[k]), kLog2e, c));
-            w[k] = pack_bf16x2(lo, hi) ^ sign2;
-        }
-        q[j] = make_uint4(w[0], w[1], w[2], w[3]);
-    }
-}
+constexpr int kZeroThreads = 128;
+constexpr int kZeroBuf = 16384;
 
 __device__ __forceinline__ uint16_t float_to_bf16_bits(float x) {
     return (uint16_t)(pack_bf16x2(x, 0.f) & 0xffffu);
 }
 
-// one row, bf16
-__device__ __forceinline__ void dz_row_bf16(const uint16_t* zrow, uint16_t* orow, int vocab, int y,
-                                            float c, float g) {
-    constexpr int U = 4;
-    const int tid = threadIdx.x;
-    const int nvec = vocab >> 3;
-    const uint4* rv = reinterpret_cast<const uint4*>(zrow);
-    uint4* ov = reinterpret_cast<uint4*>(orow);
-    const uint32_t sign2 = (g < 0.f) ? 0x80008000u : 0u;
-    const int yv = y >> 3;
+struct RowConstBf16 {
+    float c;         // -lse log2(e) + log2|g|
+    float g;         // coefficient
+    uint32_t sign2;  // sign of g on both halves of a packed pair
+    int y;
+};
+struct RowConstF32 {
+    float M, a, g;  // row max, lse - M, coefficient
+    int y;
+};
 
-    auto fix_target = [&](uint4& q, const uint4& zq) {
-        // the sampled token's entry is g (p_y - 1): recompute it in float from the logit
-        const uint32_t zw[4] = {zq.x, zq.y, zq.z, zq.w};
-        uint32_t ow[4] = {q.x, q.y, q.z, q.w};
-        const int k = (y & 7) >> 1;
-        const bool hi = (y & 1) != 0;
-        const float z = hi ? bf16_hi(zw[k]) : bf16_lo(zw[k]);
-        const float p_scaled = ex2_approx(fmaf(z, kLog2e, c));  // |g| p_y
-        const float val = (g < 0.f ? -p_scaled : p_scaled) - g;
-        const uint32_t b = float_to_bf16_bits(val);
-        ow[k] = hi ? ((ow[k] & 0x0000ffffu) | (b << 16)) : ((ow[k] & 0xffff0000u) | b);
-        q = make_uint4(ow[0], ow[1], ow[2], ow[3]);
-    };
-
-    int v = tid;
-    for (; v + (U - 1) * kThreads < nvec; v += U * kThreads) {
-        uint4 z[U], q[U];
+// one 16-byte vector of bf16 logits -> dlogits; `e0` is the column of its first element
+__device__ __forceinline__ uint4 dz_vec(uint4 z, int e0, const RowConstBf16& rc) {
+    uint32_t w[4] = {z.x, z.y, z.z, z.w};
 #pragma unroll
-        for (int j = 0; j < U; ++j) q[j] = z[j] = ld_stream(rv + v + j * kThreads);
-        dz_batch_bf16<U>(q, c, sign2);
-#pragma unroll
-        for (int j = 0; j < U; ++j) {
-            if (v + j * kThreads == yv) fix_target(q[j], z[j]);
-            st_stream(ov + v + j * kThreads, q[j]);
+    for (int k = 0; k < 4; ++k) {
+        float lo = ex2_approx(fmaf(bf16_lo(w[k]), kLog2e, rc.c));
+        float hi = ex2_approx(fmaf(bf16_hi(w[k]), kLog2e, rc.c));
+        uint32_t out = pack_bf16x2(lo, hi) ^ rc.sign2;
+        // the sampled token's entry is g (p_y - 1), formed in float before rounding
+        if (e0 + 2 * k == (rc.y & ~1)) {
+            const float ps = (rc.y & 1) ? hi : lo;
+            const float val = (rc.g < 0.f ? -ps : ps) - rc.g;
+            const uint32_t b = float_to_bf16_bits(val);
+            out = (rc.y & 1) ? ((out & 0x0000ffffu) | (b << 16)) : ((out & 0xffff0000u) | b);
         }
+        w[k] = out;
     }
-    for (; v < nvec; v += kThreads) {
-        uint4 z[1], q[1];
-        q[0] = z[0] = ld_stream(rv + v);
-        dz_batch_bf16<1>(q, c, sign2);
-        if (v == yv) fix_target(q[0], z[0]);
-        st_stream(ov + v, q[0]);
-    }
-    const int e = (nvec << 3) + tid;
-    if (e < vocab) {
-        const float z = __uint_as_float(((uint32_t)zrow[e]) << 16);
-        const float ps = ex2_approx(fmaf(z, kLog2e, c));
-        float val = (g < 0.f) ? -ps : ps;
-        if (e == y) val -= g;
-        orow[e] = float_to_bf16_bits(val);
-    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
-// one row, fp32
-__device__ __forceinline__ void dz_row_f32(const float* zrow, float* orow, int vocab, int y, float M,
-                                           float a, float g) {
-    constexpr int U = 4;
-    const int tid = threadIdx.x;
-    const int nvec = vocab >> 2;
-    const float4* rv = reinterpret_cast<const float4*>(zrow);
-    float4* ov = reinterpret_cast<float4*>(orow);
-    const int yv = y >> 2;
-    auto one = [&](float z) { return g * expf((z - M) - a); };
-    auto vec = [&](float4 z, int vi) {
-        float4 o = make_float4(one(z.x), one(z.y), one(z.z), one(z.w));
-        if (vi == yv) {
-            const int k = y & 3;
-            if (k == 0) o.x -= g;
-            else if (k == 1) o.y -= g;
-            else if (k == 2) o.z -= g;
-            else o.w -= g;
-        }
-        return o;
-    };
-    int v = tid;
-    for (; v + (U - 1) * kThreads < nvec; v += U * kThreads) {
-        float4 z[U];
+__device__ __forceinline__ uint4 dz_vec(uint4 zbits, int e0, const RowConstF32& rc) {
+    float z[4] = {__uint_as_float(zbits.x), __uint_as_float(zbits.y), __uint_as_float(zbits.z),
+                  __uint_as_float(zbits.w)};
+    uint32_t o[4];
 #pragma unroll
-        for (int j = 0; j < U; ++j) z[j] = __ldcs(rv + v + j * kThreads);
-#pragma unroll
-        for (int j = 0; j < U; ++j) __stcs(ov + v + j * kThreads, vec(z[j], v + j * kThreads));
+    for (int k = 0; k < 4; ++k) {
+        float v = rc.g * expf((z[k] - rc.M) - rc.a);
+        if (e0 + k == rc.y) v -= rc.g;
+        o[k] = __float_as_uint(v);
     }
-    for (; v < nvec; v += kThreads) __stcs(ov + v, vec(__ldcs(rv + v), v));
-    const int e = (nvec << 2) + tid;
-    if (e < vocab) {
-        float val = one(zrow[e]);
-        if (e == y) val -= g;
-        orow[e] = val;
-    }
+    return make_uint4(o[0], o[1], o[2], o[3]);
 }
+
+// scalar tail elements (vocab not a multiple of the vector width): read from the stage, written
+// straight to global memory
+__device__ __forceinline__ void dz_scalar(const void* zsm, void* orow, int e_in_chunk, int e,
+                                          const RowConstBf16& rc) {
+    const float z = __uint_as_float(((uint32_t) static_cast<const uint16_t*>(zsm)[e_in_chunk]) << 16);
+    const float ps = ex2_approx(fmaf(z, kLog2e, rc.c));
+    float val = (rc.g < 0.f) ? -ps : ps;
+    if (e == rc.y) val -= rc.g;
+    static_cast<uint16_t*>(orow)[e] = float_to_bf16_bits(val);
+}
+__device__ __forceinline__ void dz_scalar(const void* zsm, void* orow, int e_in_chunk, int e,
+                                          const RowConstF32& rc) {
+    const float z = static_cast<const float*>(zsm)[e_in_chunk];
+    float val = rc.g * expf((z - rc.M) - rc.a);
+    if (e == rc.y) val -= rc.g;
+    static_cast<float*>(orow)[e] = val;
+}
+
+__device__ __forceinline__ void consumer_barrier() {
+    asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory");
+}
+
+__device__ __forceinline__ bool row_is_live(const Workspace& ws, int64_t r, int seq_len) {
+    return ws.row_state[r] == ROW_OK && ws.coef[(int)(r / seq_len)] != 0.0;
+}
+
+// ---- dead rows ------------------------------------------------------------------------------------
 
 template <int ESIZE>
-__device__ __forceinline__ void zero_row(void* orow, int vocab) {
+__global__ void __launch_bounds__(kZeroThreads)
+zero_rows_kernel(void* dlogits, int64_t ld, int vocab, int seq_len, int64_t row0, int64_t n_rows,
+                 Workspace ws) {
+    __shared__ __align__(128) uint8_t zeros[kZeroBuf];
     const int tid = threadIdx.x;
-    constexpr int per = 16 / ESIZE;
-    const int nvec = vocab / per;
-    uint4* ov = reinterpret_cast<uint4*>(orow);
-    for (int v = tid; v < nvec; v += kThreads) st_stream(ov + v, make_uint4(0, 0, 0, 0));
-    const int e = nvec * per + tid;
-    if (e < vocab) {
-        if (ESIZE == 2) static_cast<uint16_t*>(orow)[e] = 0;
-        else static_cast<float*>(orow)[e] = 0.f;
+    for (int i = tid; i < kZeroBuf / 16; i += kZeroThreads)
+        reinterpret_cast<uint4*>(zeros)[i] = make_uint4(0, 0, 0, 0);
+    fence_proxy_async_smem();
+    __syncthreads();
+    const int whole = (vocab * ESIZE) / 16 * 16;  // bytes of a row in whole 16-byte vectors
+    const int tail0 = whole / ESIZE;              // first column not covered by them
+    for (int64_t i = blockIdx.x; i < n_rows; i += gridDim.x) {
+        const int64_t r = row0 + i;
+        if (row_is_live(ws, r, seq_len)) continue;
+        uint8_t* orow = static_cast<uint8_t*>(dlogits) + (size_t)i * ld * ESIZE;
+        if (tid == 0) {
+            for (int o = 0; o < whole; o += kZeroBuf) bulk_store(orow + o, zeros, (uint32_t)min(kZeroBuf, whole - o));
+            bulk_commit();
+        } else if (tail0 + (tid - 1) < vocab) {  // fewer than 16 bytes of ragged tail
+            if (ESIZE == 2) reinterpret_cast<uint16_t*>(orow)[tail0 + tid - 1] = 0;
+            else reinterpret_cast<float*>(orow)[tail0 + tid - 1] = 0.f;
+        }
     }
+    if (tid == 0) bulk_wait_all<0>();  // the zero buffer must outlive every copy that reads it
 }
+
+// ---- live rows ------------------------------------------------------------------------------------
 
 template <int DT>
 __global__ void __launch_bounds__(kThreads)
 dlogits_kernel(const void* logits, void* dlogits /* may alias logits */, int64_t ld, int vocab,
                int seq_len, int64_t row0, int64_t n_rows, const int32_t* __restrict__ targets,
-               Workspace ws) {
-    for (int64_t i = blockIdx.x; i < n_rows; i += gridDim.x) {
-        const int64_t r = row0 + i;
-        const int n = (int)(r / seq_len);
-        const double g = ws.coef[n];
-        const bool live = (ws.row_state[r] == ROW_OK) && (g != 0.0);
-        if (DT == RAPID_BF16) {
-            uint16_t* orow = static_cast<uint16_t*>(dlogits) + i * ld;
-            if (!live) {
-                zero_row<2>(orow, vocab);
-                continue;
-            }
-            const float c = (float)fma(-ws.lse[r], kLog2eD, ws.coef_log2[n]);
-            dz_row_bf16(static_cast<const uint16_t*>(logits) + i * ld, orow, vocab, targets[r], c,
-                        (float)g);
-        } else {
-            float* orow = static_cast<float*>(dlogits) + i * ld;
-            if (!live) {
-                zero_row<4>(orow, vocab);
-                continue;
-            }
-            const float M = ws.row_max[r];
-            const float a = (float)(ws.lse[r] - (double)M);
-            dz_row_f32(static_cast<const float*>(logits) + i * ld, orow, vocab, targets[r], M, a,
-                       (float)g);
+               rapid_stats_t* stats_user, Workspace ws) {
+    constexpr int ESIZE = (DT == RAPID_BF16) ? 2 : 4;
+    constexpr int PER = 16 / ESIZE;  // elements per 16-byte vector
+    using RowConst = typename std::conditional<DT == RAPID_BF16, RowConstBf16, RowConstF32>::type;
+
+    extern __shared__ __align__(128) uint8_t ring[];  // kStages x kChunk
+    __shared__ __align__(8) uint64_t full_bar[kStages];
+    __shared__ __align__(8) uint64_t empty_bar[kStages];
+    __shared__ int abort_flag;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], 1);
         }
+        abort_flag = 0;
+        mbar_init_fence();
     }
+    __syncthreads();
+    volatile int* abortp = &abort_flag;
+
+    // bytes of a row that are loaded: the vocabulary rounded up to whole 16-byte vectors (the
+    // pitch is a multiple of 16 bytes and >= vocab, so this stays inside the row); bytes that are
+    // stored in bulk: the whole vectors of real columns only
+    const int load_bytes = ((vocab * ESIZE + 15) / 16) * 16;
+    const int n_chunks = (load_bytes + kChunk - 1) / kChunk;
+    const int nvec_row = vocab / PER;
+
+    if (warp == kConsumerWarps) {
+        // ------------------------------- producer -------------------------------------------
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int64_t i = blockIdx.x; i < n_rows && ok; i += gridDim.x) {
+                if (!row_is_live(ws, row0 + i, seq_len)) continue;
+                const uint8_t* src = static_cast<const uint8_t*>(logits) + (size_t)i * ld * ESIZE;
+                for (int c = 0; c < n_chunks; ++c, ++it) {
+                    const int s = it % kStages;
+                    const uint32_t use = it / kStages;
+                    if (use > 0 && !mbar_wait_bounded(&empty_bar[s], (use & 1u) ^ 1u, abortp)) {
+                        ok = false;
+                        break;
+                    }
+                    const int bytes = min(kChunk, load_bytes - c * kChunk);
+                    mbar_arrive_expect_tx(&full_bar[s], (uint32_t)bytes);
+                    bulk_load(ring + (size_t)s * kChunk, src + (size_t)c * kChunk, (uint32_t)bytes,
+                              &full_bar[s]);
+                }
+            }
+            if (!ok || *abortp) {
+                // gave up: let the copies already issued land before the CTA's memory goes away
+                const uint32_t first = it > (uint32_t)kStages ? it - kStages : 0u;
+                for (uint32_t j = first; j < it; ++j) {
+                    const unsigned long long t0 = global_timer_ns();
+                    while (!mbar_try_wait(&full_bar[j % kStages], (j / kStages) & 1u))
+                        if (global_timer_ns() - t0 > kWaitLimitNs) break;
+                }
+            }
+        }
+    } else {
+        // ------------------------------- consumers ------------------------------------------
+        uint32_t it = 0;
+        bool ok = true;
+        for (int64_t i = blockIdx.x; i < n_rows && ok; i += gridDim.x) {
+            const int64_t r = row0 + i;
+            if (!row_is_live(ws, r, seq_len)) continue;
+            const int n = (int)(r / seq_len);
+            const double g = ws.coef[n];
+            uint8_t* orow = static_cast<uint8_t*>(dlogits) + (size_t)i * ld * ESIZE;
+            RowConst rc;
+            if constexpr (DT == RAPID_BF16) {
+                rc.c = (float)fma(-ws.lse[r], kLog2eD, ws.coef_log2[n]);
+                rc.g = (float)g;
+                rc.sign2 = (g < 0.0) ? 0x80008000u : 0u;
+                rc.y = targets[r];
+            } else {
+                rc.M = ws.row_max[r];
+                rc.a = (float)(ws.lse[r] - (double)rc.M);
+                rc.g = (float)g;
+                rc.y = targets[r];
+            }
+            for (int c = 0; c < n_chunks; ++c, ++it) {
+                const int s = it % kStages;
+                // A wait that gives up raises the abort flag; the thread still goes to the barrier
+                // below, after which every consumer sees the flag and leaves together.
+                const bool got = mbar_wait_bounded(&full_bar[s], (it / kStages) & 1u, abortp);
+                uint4* sv = reinterpret_cast<uint4*>(ring + (size_t)s * kChunk);
+                const int v0 = c * kVecPerChunk;                  // first vector of the chunk in the row
+                const int nv = min(kVecPerChunk, nvec_row - v0);  // whole real vectors in the chunk
+                if (got) {
+                    // ragged tail of the row (fewer than one vector of real columns), before the
+                    // stage is overwritten
+                    if (c == n_chunks - 1) {
+                        const int e = nvec_row * PER + tid;
+                        if (e < vocab) dz_scalar(sv, orow, e - v0 * PER, e, rc);
+                    }
+                    uint4 z[kVecPerThread];
+#pragma unroll
+                    for (int j = 0; j < kVecPerThread; ++j) {
+                        const int v = tid + j * kConsumers;
+                        if (v < nv) z[j] = sv[v];
+                    }
+#pragma unroll
+                    for (int j = 0; j < kVecPerThread; ++j) {
+                        const int v = tid + j * kConsumers;
+                        if (v < nv) sv[v] = dz_vec(z[j], (v0 + v) * PER, rc);
+                    }
+                    fence_proxy_async_smem();  // generic writes above -> asynchronous read below
+                }
+                consumer_barrier();
+                if (*abortp) {
+                    ok = false;
+                    break;
+                }
+                if (tid == 0) {
+                    if (nv > 0) bulk_store(orow + (size_t)c * kChunk, sv, (uint32_t)nv * 16u);
+                    bulk_commit();
+                    // the store committed kStoreDepth chunks ago has finished reading its stage
+                    bulk_wait_read<kStoreDepth>();
+                    if (it >= (uint32_t)kStoreDepth) mbar_arrive(&empty_bar[(it - kStoreDepth) % kStages]);
+                }
+            }
+        }
+        if (tid == 0) bulk_wait_all<0>();
+    }
+    __syncthreads();
+    if (tid == 0 && abort_flag) {
+        atomicMax(&ws.stats->status, (int)RAPID_ERR_TIMEOUT);
+        if (stats_user) atomicMax(&stats_user->status, (int)RAPID_ERR_TIMEOUT);
+    }
+}
+
+template <int DT>
+cudaError_t launch_one(const rapid_desc_t& d, const void* logits_chunk, void* dlogits_chunk,
+                       int64_t row0, int64_t n_rows, const int32_t* targets, rapid_stats_t* stats_user,
+                       const Workspace& ws, int sm_count, cudaStream_t stream) {
+    constexpr int ESIZE = (DT == RAPID_BF16) ? 2 : 4;
+    // dead rows first: a pure write stream
+    {
+        int64_t grid = (int64_t)sm_count * 16;
+        if (grid > n_rows) grid = n_rows;
+        zero_rows_kernel<ESIZE><<<(unsigned)grid, kZeroThreads, 0, stream>>>(dlogits_chunk, d.ld, d.vocab,
+                                                                             d.seq_len, row0, n_rows, ws);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    constexpr size_t smem = (size_t)kStages * kChunk;
+    cudaError_t e = cudaFuncSetAttribute(dlogits_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)smem);
+    if (e != cudaSuccess) return e;
+    int per_sm = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dlogits_kernel<DT>, kThreads, smem);
+    if (e != cudaSuccess) return e;
+    if (per_sm < 1) per_sm = 1;
+    int64_t grid = (int64_t)sm_count * per_sm;
+    if (grid > n_rows) grid = n_rows;
+    dlogits_kernel<DT><<<(unsigned)grid, kThreads, smem, stream>>>(
+        logits_chunk, dlogits_chunk, d.ld, d.vocab, d.seq_len, row0, n_rows, targets, stats_user, ws);
+    return cudaGetLastError();
 }
 
 }  // namespace
 
 cudaError_t launch_dlogits(const rapid_desc_t& d, const void* logits_chunk, void* dlogits_chunk,
                            int64_t row0, int64_t n_rows, const int32_t* targets,
-                           const Workspace& ws, int sm_count, cudaStream_t stream) {
+                           rapid_stats_t* stats_user, const Workspace& ws, int sm_count,
+                           cudaStream_t stream) {
     if (n_rows <= 0) return cudaSuccess;
-    int per_sm = 0;
-    cudaError_t e;
     if (d.dtype == RAPID_BF16)
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dlogits_kernel<RAPID_BF16>,
-                                                          kThreads, 0);
-    else
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dlogits_kernel<RAPID_F32>,
-                                                          kThreads, 0);
-    if (e != cudaSuccess) return e;
-    if (per_sm < 1) per_sm = 1;
-    int64_t grid = (int64_t)sm_count * per_sm;
-    if (grid > n_rows) grid = n_rows;
-    if (d.dtype == RAPID_BF16)
-        dlogits_kernel<RAPID_BF16><<<(unsigned)grid, kThreads, 0, stream>>>(
-            logits_chunk, dlogits_chunk, d.ld, d.vocab, d.seq_len, row0, n_rows, targets, ws);
-    else
-        dlogits_kernel<RAPID_F32><<<(unsigned)grid, kThreads, 0, stream>>>(
-            logits_chunk, dlogits_chunk, d.ld, d.vocab, d.seq_len, row0, n_rows, targets, ws);
-    return cudaGetLastError();
+        return launch_one<RAPID_BF16>(d, logits_chunk, dlogits_chunk, row0, n_rows, targets, stats_user,
+                                      ws, sm_count, stream);
+    return launch_one<RAPID_F32>(d, logits_chunk, dlogits_chunk, row0, n_rows, targets, stats_user, ws,
+                                 sm_count, stream);
 }
 
 }  // namespace rapid

@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <type_traits>
+
 #include "rapid_pg.h"
 
 namespace rapid {
@@ -139,6 +141,7 @@ cudaError_t launch_group_advantage(const rapid_desc_t& d, const float* rewards,
                                    cudaStream_t stream);
 cudaError_t launch_dlogits(const rapid_desc_t& d, const void* logits_chunk, void* dlogits_chunk,
                            int64_t row0, int64_t n_rows, const int32_t* targets,
-                           const Workspace& ws, int sm_count, cudaStream_t stream);
+                           rapid_stats_t* stats_user, const Workspace& ws, int sm_count,
+                           cudaStream_t stream);
 
 }  // namespace rapid

@@ -78,7 +78,7 @@ def test_config_long_scaled_chunked():
     for r0 in starts:
         n = min(chunk, T - r0)
         zc = b["logits"][r0:r0 + n].to(dev)
-        rb.rapid_pg_dlogits_chunk(desc, zc, dz[r0:r0 + n], r0, n, tg, ws)
+        rb.rapid_pg_dlogits_chunk(desc, zc, dz[r0:r0 + n], r0, n, tg, st, ws)
     torch.cuda.synchronize()
     g2 = {"loss": loss.item(), "token_logp": tl.cpu().numpy(), "adv": adv.cpu().numpy(),
           "stats": rb.read_stats(st), "dlogits": dz.cpu().numpy()}

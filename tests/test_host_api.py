@@ -100,7 +100,7 @@ def test_chunk_range_validation():
     big = 1 << 40
     assert L.rapid_pg_stats_chunk(C.byref(d), FAKE, 30, 3, FAKE, None, FAKE, big, None) == rb.RAPID_ERR_INVALID_ARG
     assert L.rapid_pg_stats_chunk(C.byref(d), FAKE, -1, 3, FAKE, None, FAKE, big, None) == rb.RAPID_ERR_INVALID_ARG
-    assert L.rapid_pg_dlogits_chunk(C.byref(d), FAKE, FAKE + 256, 0, 8, FAKE, FAKE, big, None) == rb.RAPID_ERR_INVALID_ARG
+    assert L.rapid_pg_dlogits_chunk(C.byref(d), FAKE, FAKE + 256, 0, 8, FAKE, None, FAKE, big, None) == rb.RAPID_ERR_INVALID_ARG
     assert L.rapid_group_advantage(C.byref(d), None, None, FAKE, FAKE, None, None, None) == rb.RAPID_ERR_INVALID_ARG
 
 
