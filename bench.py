@@ -326,7 +326,7 @@ def run_ours(args):
                    "eta": 2.0, "parallelism": f"dp{world} (by prompt group, no data-path collective)"},
         "clocks": clocks,
         "e2e": e2e,
-        "gpu_launches": 4 * args.steps,
+        "gpu_launches": 5 * args.steps,
         "roofline": {"bound": "hbm", "kernel": "dlogits_kernel (pass 2)", "achieved": ach_p2,
                      "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": ach_p2 / peak,
                      "frac_of_8TBs_nominal": ach_p2 / 8000.0, "ms_per_launch": p2,
