@@ -166,6 +166,41 @@ rapid_status_t rapid_pg_loss_fwd_bwd(const rapid_desc_t* desc, const void* logit
                                      void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * rapid_pg_loss_fwd_bwd without a caller-provided workspace.  (The paper has no counterpart to
+ * this call; it exists for deployment reasons only.)
+ *
+ * Some users of this library are not in a position to allocate device memory for the workspace:
+ * a plug-in inside a host application whose memory pool already owns the whole device and
+ * forbids allocations behind its back; a serving or training loop that has handed out its entire
+ * memory budget up front and treats any later allocation as a bug; a latency-critical loop that
+ * cannot afford the device-wide stall an allocation may cause.  For them the scratch memory is a
+ * fixed array of RAPID_NOALLOC_SCRATCH_BYTES inside the library's device image.  Every GPU on
+ * which the library is loaded holds that array until the process exits.
+ *
+ * Arguments and results are exactly those of rapid_pg_loss_fwd_bwd, minus the workspace; the
+ * caller still owns and passes every input and output array.
+ *
+ *   - Limit: the problem must satisfy rapid_workspace_bytes(desc) <= RAPID_NOALLOC_SCRATCH_BYTES
+ *     (about 21 bytes per row of the token grid, i.e. up to roughly 199 000 rows).  Anything
+ *     larger returns RAPID_ERR_UNSUPPORTED and enqueues nothing; use the workspace form instead.
+ *   - The call allocates and frees nothing, on the device or through any library.
+ *   - First call on each device: the library looks up the device address of its array (a
+ *     cudaGetSymbolAddress call, made with the caller's current device) and remembers it.  Make
+ *     this first call, on every device you will use, before beginning any stream capture.
+ *   - All calls on a device share the one array, and it keeps whatever the previous call left in
+ *     it.  Nothing in it needs clearing between calls (each call rewrites what it reads), but two
+ *     calls whose GPU work can overlap -- different streams, or different host threads without
+ *     ordering between their streams -- race on it and give undefined results.  Serialise them.
+ */
+#define RAPID_NOALLOC_SCRATCH_BYTES (4u << 20)
+rapid_status_t rapid_pg_loss_fwd_bwd_noalloc(const rapid_desc_t* desc, const void* logits,
+                                             const int32_t* targets, const uint8_t* mask,
+                                             const float* behav_logp, const float* rewards,
+                                             const int32_t* group_offsets, void* dlogits,
+                                             float* loss, float* token_logp, float* adv,
+                                             rapid_stats_t* stats, void* stream);
+
+/*
  * The same path in three steps, for logits that are produced (or fit in memory) only a block of
  * rows at a time.  The order is forced by the data: every generation of a group must have gone
  * through the statistics pass before any of the group's dlogits can be written.

@@ -38,6 +38,7 @@ FLAG_LOO_LITERAL_DIVISOR = 16
 EXPORTS = (
     "rapid_status_string", "rapid_version", "rapid_workspace_bytes", "rapid_group_advantage",
     "rapid_pg_loss_fwd_bwd", "rapid_pg_stats_chunk", "rapid_pg_finalize", "rapid_pg_dlogits_chunk",
+    "rapid_pg_loss_fwd_bwd_noalloc",
 )
 
 
@@ -85,6 +86,8 @@ def lib():
         L.rapid_group_advantage.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp]
         L.rapid_pg_loss_fwd_bwd.restype = C.c_int
         L.rapid_pg_loss_fwd_bwd.argtypes = [dp] + [vp] * 12 + [sz, vp]
+        L.rapid_pg_loss_fwd_bwd_noalloc.restype = C.c_int
+        L.rapid_pg_loss_fwd_bwd_noalloc.argtypes = [dp] + [vp] * 12
         L.rapid_pg_stats_chunk.restype = C.c_int
         L.rapid_pg_stats_chunk.argtypes = [dp, vp, i64, i64, vp, vp, vp, sz, vp]
         L.rapid_pg_finalize.restype = C.c_int
@@ -169,6 +172,24 @@ def rapid_pg_loss_fwd_bwd(desc: RapidDesc, logits: torch.Tensor, targets: torch.
         C.byref(desc), _ptr(logits), _ptr(targets), _ptr(mask), _ptr(behav_logp), _ptr(rewards),
         _ptr(group_offsets), _ptr(dlogits), _ptr(loss), _ptr(token_logp), _ptr(adv), _ptr(stats),
         _ptr(workspace), workspace.numel(), _stream()), "rapid_pg_loss_fwd_bwd")
+
+
+NOALLOC_SCRATCH_BYTES = 4 << 20
+
+
+def rapid_pg_loss_fwd_bwd_noalloc(desc: RapidDesc, logits: torch.Tensor, targets: torch.Tensor,
+                                  mask: Optional[torch.Tensor], behav_logp: torch.Tensor,
+                                  rewards: torch.Tensor, group_offsets: torch.Tensor,
+                                  dlogits: torch.Tensor, loss: torch.Tensor,
+                                  token_logp: Optional[torch.Tensor], adv: Optional[torch.Tensor],
+                                  stats: Optional[torch.Tensor]) -> None:
+    """rapid_pg_loss_fwd_bwd for callers that cannot allocate a workspace: the scratch is a fixed
+    array inside the library (at most NOALLOC_SCRATCH_BYTES; larger problems raise
+    RAPID_ERR_UNSUPPORTED).  Calls on one device share that array, so do not let two overlap."""
+    _check(lib().rapid_pg_loss_fwd_bwd_noalloc(
+        C.byref(desc), _ptr(logits), _ptr(targets), _ptr(mask), _ptr(behav_logp), _ptr(rewards),
+        _ptr(group_offsets), _ptr(dlogits), _ptr(loss), _ptr(token_logp), _ptr(adv), _ptr(stats),
+        _stream()), "rapid_pg_loss_fwd_bwd_noalloc")
 
 
 def rapid_pg_stats_chunk(desc: RapidDesc, logits_chunk: torch.Tensor, row0: int, n_rows: int,
