@@ -18,6 +18,15 @@ LOGP_ATOL = {torch.float32: 2e-6, torch.bfloat16: 2e-5}
 ADV_ATOL = {torch.float32: 2e-6, torch.bfloat16: 2e-4}
 
 
+def adv_atol(dtype, seq_len: int) -> float:
+    """Advantages of the whole path depend on w_n = exp(sum of up to seq_len token log-probs).
+    With float32 logits each row's log-sum-exp carries a few 1e-9 of error (float32 exponentials
+    and differences, averaged over the vocabulary), which adds up over the generation; the
+    advantage inherits it through mean(c R) with c <= eta = 2.  So the bound grows with L."""
+    per_token = 4e-9 if dtype == torch.float32 else 4e-7
+    return max(ADV_ATOL[dtype], per_token * seq_len)
+
+
 def loss_scale(o) -> float:
     """The loss is a signed sum; its relative error is measured against
     max(|loss|, 1e-3 * sum_n |g_n S_n|)."""
@@ -101,7 +110,7 @@ def compare(o, g, dtype, seq_len, check_dlogits=True):
     ok = o["row_ok"].astype(bool)
     np.testing.assert_allclose(g["token_logp"], o["token_logp"], rtol=0, atol=LOGP_ATOL[dtype])
     assert np.all(g["token_logp"][~ok] == 0.0)
-    np.testing.assert_allclose(g["adv"], o["adv64"], rtol=0, atol=ADV_ATOL[dtype])
+    np.testing.assert_allclose(g["adv"], o["adv64"], rtol=0, atol=adv_atol(dtype, seq_len))
     rel = abs(g["loss"] - o["loss"]) / loss_scale(o)
     # the float32 loss output itself carries half an ulp
     assert rel <= LOSS_RTOL[dtype] + 6e-8 * abs(o["loss"]) / loss_scale(o), f"loss rel err {rel}"
