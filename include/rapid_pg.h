@@ -236,6 +236,46 @@ rapid_status_t rapid_pg_dlogits_chunk(const rapid_desc_t* desc, const void* logi
                                       const int32_t* targets, rapid_stats_t* stats,
                                       void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * The fused LM-head form: the logits z = hidden * w_vocab are formed tile by tile on the tensor
+ * cores and never written to memory (this form comes from the benchmark definition; in the paper
+ * the logits are simply the policy network's output, Sec. 3.1).  Computes the same loss as
+ * rapid_pg_loss_fwd_bwd on z, and the gradients with respect to both factors:
+ *     dhidden = dlogits * w_vocab^T,      dW = hidden^T * dlogits,
+ * where dlogits (as defined at the top of this file) is rounded to bf16 before these two products.
+ *
+ *   desc        dtype must be RAPID_BF16; desc->ld is the row pitch, in elements, of BOTH w_vocab
+ *               and dW (>= vocab, a multiple of 8)
+ *   hidden_dim  D, a multiple of 8
+ *   hidden      [T, D] bf16, contiguous rows (pitch D), 16-byte aligned
+ *   w_vocab     [D, ld] bf16, 16-byte aligned
+ *   targets, mask, behav_logp, rewards, group_offsets: as for rapid_pg_loss_fwd_bwd
+ *   loss        [1] float out
+ *   dhidden     [T, D] bf16 out (pitch D); rows that are masked or have g_n = 0 come out as zeros
+ *   dW          [D, ld] float out.  Stores go out in 16-byte units: when vocab is not a multiple
+ *               of 4, the columns from vocab up to the next multiple of 4 are written as zeros;
+ *               columns beyond that are untouched
+ *   token_logp, adv, stats: optional outputs as for rapid_pg_loss_fwd_bwd
+ *   workspace   rapid_fused_head_workspace_bytes(desc, hidden_dim) bytes, 1024-byte aligned.  It
+ *               holds, besides the per-row state, one bf16 copy of dlogits ([T, vocab] rounded up
+ *               to 64 columns) and two floats per row per 256 vocabulary columns.
+ *
+ * Four tensor-core kernels run (forward statistics, dlogits, dhidden, dW), each a persistent grid
+ * with bounded waits: a wait that gives up raises stats->status to RAPID_ERR_TIMEOUT and leaves the
+ * outputs unspecified.  Returns RAPID_ERR_CUDA if the driver cannot encode the tensor maps.
+ */
+rapid_status_t rapid_fused_head_workspace_bytes(const rapid_desc_t* desc, int32_t hidden_dim,
+                                                size_t* bytes);
+
+rapid_status_t rapid_pg_loss_fused_head(const rapid_desc_t* desc, int32_t hidden_dim,
+                                        const void* hidden, const void* w_vocab,
+                                        const int32_t* targets, const uint8_t* mask,
+                                        const float* behav_logp, const float* rewards,
+                                        const int32_t* group_offsets, float* loss, void* dhidden,
+                                        void* dW, float* token_logp, float* adv,
+                                        rapid_stats_t* stats, void* workspace,
+                                        size_t workspace_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -38,7 +38,7 @@ FLAG_LOO_LITERAL_DIVISOR = 16
 EXPORTS = (
     "rapid_status_string", "rapid_version", "rapid_workspace_bytes", "rapid_group_advantage",
     "rapid_pg_loss_fwd_bwd", "rapid_pg_stats_chunk", "rapid_pg_finalize", "rapid_pg_dlogits_chunk",
-    "rapid_pg_loss_fwd_bwd_noalloc",
+    "rapid_pg_loss_fwd_bwd_noalloc", "rapid_fused_head_workspace_bytes", "rapid_pg_loss_fused_head",
 )
 
 
@@ -88,6 +88,10 @@ def lib():
         L.rapid_pg_loss_fwd_bwd.argtypes = [dp] + [vp] * 12 + [sz, vp]
         L.rapid_pg_loss_fwd_bwd_noalloc.restype = C.c_int
         L.rapid_pg_loss_fwd_bwd_noalloc.argtypes = [dp] + [vp] * 12
+        L.rapid_fused_head_workspace_bytes.restype = C.c_int
+        L.rapid_fused_head_workspace_bytes.argtypes = [dp, C.c_int32, C.POINTER(C.c_size_t)]
+        L.rapid_pg_loss_fused_head.restype = C.c_int
+        L.rapid_pg_loss_fused_head.argtypes = [dp, C.c_int32] + [vp] * 14 + [sz, vp]
         L.rapid_pg_stats_chunk.restype = C.c_int
         L.rapid_pg_stats_chunk.argtypes = [dp, vp, i64, i64, vp, vp, vp, sz, vp]
         L.rapid_pg_finalize.restype = C.c_int
@@ -217,6 +221,35 @@ def rapid_pg_dlogits_chunk(desc: RapidDesc, logits_chunk: torch.Tensor,
     _check(lib().rapid_pg_dlogits_chunk(C.byref(desc), _ptr(logits_chunk), _ptr(dlogits_chunk),
                                         row0, n_rows, _ptr(targets), _ptr(stats), _ptr(workspace),
                                         workspace.numel(), _stream()), "rapid_pg_dlogits_chunk")
+
+
+def rapid_fused_head_workspace_bytes(desc: RapidDesc, hidden_dim: int) -> int:
+    n = C.c_size_t(0)
+    _check(lib().rapid_fused_head_workspace_bytes(C.byref(desc), int(hidden_dim), C.byref(n)),
+           "rapid_fused_head_workspace_bytes")
+    return int(n.value)
+
+
+def alloc_fused_head_workspace(desc: RapidDesc, hidden_dim: int, device="cuda") -> torch.Tensor:
+    """Device scratch for rapid_pg_loss_fused_head, on a 1024-byte boundary."""
+    n = rapid_fused_head_workspace_bytes(desc, hidden_dim)
+    buf = torch.empty(n + 1024, dtype=torch.uint8, device=device)
+    off = (-buf.data_ptr()) % 1024
+    return buf[off:off + n]
+
+
+def rapid_pg_loss_fused_head(desc: RapidDesc, hidden: torch.Tensor, w_vocab: torch.Tensor,
+                             targets: torch.Tensor, mask: Optional[torch.Tensor],
+                             behav_logp: torch.Tensor, rewards: torch.Tensor,
+                             group_offsets: torch.Tensor, loss: torch.Tensor, dhidden: torch.Tensor,
+                             dW: torch.Tensor, token_logp: Optional[torch.Tensor],
+                             adv: Optional[torch.Tensor], stats: Optional[torch.Tensor],
+                             workspace: torch.Tensor) -> None:
+    _check(lib().rapid_pg_loss_fused_head(
+        C.byref(desc), int(hidden.shape[1]), _ptr(hidden), _ptr(w_vocab), _ptr(targets), _ptr(mask),
+        _ptr(behav_logp), _ptr(rewards), _ptr(group_offsets), _ptr(loss), _ptr(dhidden), _ptr(dW),
+        _ptr(token_logp), _ptr(adv), _ptr(stats), _ptr(workspace), workspace.numel(), _stream()),
+        "rapid_pg_loss_fused_head")
 
 
 @dataclass

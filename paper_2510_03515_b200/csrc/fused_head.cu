@@ -1,0 +1,439 @@
+// The fused LM-head form of the path: the logits z = h W are never written to memory.
+//
+//   forward   z tiles are formed on the tensor cores (umma_gemm.cuh); the epilogue keeps, per row
+//             and per 256-column tile, the running maximum and the sum of exponentials, and picks
+//             out the sampled token's logit.  A small merge kernel turns the per-tile pairs into
+//             lse and log pi_theta(y_t) in double, in the same workspace layout the logits-in
+//             path uses, so the per-generation reduce and the finalize step are shared.
+//   backward  z tiles are formed again; the epilogue turns them into
+//             dz = g_n m_r (softmax - onehot) in bf16 and stores them (TMA) into a scratch
+//             matrix.  Two more GEMMs follow: dh = dz W^T (K = vocabulary) and dW = h^T dz
+//             (K = rows; both operands read MN-major straight from their row-major storage).
+//
+// Four GEMM-sized contractions in all (forward, recompute, dh, dW); only dz, in bf16, ever
+// exists in memory.
+#include <math.h>
+
+#include "rapid_common.cuh"
+#include "umma_gemm.cuh"
+
+namespace rapid {
+
+namespace {
+
+using namespace umma;
+
+// Scratch of the fused-head call, carved after the ordinary workspace.
+struct HeadScratch {
+    float* part_m;   // [n_tiles][T] running maximum of a row within one 256-column tile
+    float* part_s;   // [n_tiles][T] sum of exp(z - part_m)
+    float* zy;       // [T] the sampled token's logit
+    uint16_t* dz;    // [T][ldz] bf16
+    int* status;     // raised to RAPID_ERR_TIMEOUT by a kernel whose bounded wait ran out
+    int64_t ldz;
+    int n_tiles;
+};
+
+inline size_t carve_head(const rapid_desc_t& d, void* base, size_t off0, HeadScratch* h) {
+    const size_t T = (size_t)d.n_seq * (size_t)d.seq_len;
+    const size_t nt = ((size_t)d.vocab + BN - 1) / BN;
+    const size_t ldz = ((size_t)d.vocab + 63) / 64 * 64;
+    size_t off = off0;
+    char* p = static_cast<char*>(base);
+    auto take = [&](size_t bytes) {
+        char* q = p ? p + off : nullptr;
+        off = align_up(off + bytes, 1024);
+        return q;
+    };
+    HeadScratch s;
+    s.part_m = reinterpret_cast<float*>(take(nt * T * 4));
+    s.part_s = reinterpret_cast<float*>(take(nt * T * 4));
+    s.zy = reinterpret_cast<float*>(take(T * 4));
+    s.dz = reinterpret_cast<uint16_t*>(take(T * ldz * 2));
+    s.status = reinterpret_cast<int*>(take(256));
+    s.ldz = (int64_t)ldz;
+    s.n_tiles = (int)nt;
+    if (h) *h = s;
+    return off;
+}
+
+// ---- forward epilogue: per-tile row statistics ------------------------------------------------------
+
+struct FwdStats {
+    struct Params {
+        float* part_m;
+        float* part_s;
+        float* zy;
+        const int32_t* targets;
+        int T, V;
+    };
+    const Params& p;
+    const int row_off;  // row of this thread inside the tile
+    __device__ FwdStats(const Params& p_, uint8_t*, int quarter, int lane) : p(p_), row_off(quarter * 32 + lane) {}
+
+    __device__ void tile(int m0, int n0, uint32_t taddr) {
+        const int row = m0 + row_off;
+        const int ncols = min(BN, p.V - n0);
+        const int ycol = (row < p.T) ? (p.targets[row] - n0) : -1;
+        float m = -INFINITY, s0 = 0.f, s1 = 0.f, zyv = 0.f;
+#pragma unroll 1
+        for (int c = 0; c * 32 < ncols; ++c) {
+            uint32_t r[32];
+            tmem_ld32(taddr + c * 32, r);
+            tmem_ld_wait();
+            if (c * 32 + 32 > ncols) {  // ragged last chunk of the vocabulary: those columns do not exist
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                    if (c * 32 + j >= ncols) r[j] = 0xff800000u;  // -inf
+            }
+            float cm = __uint_as_float(r[0]);
+#pragma unroll
+            for (int j = 1; j < 32; ++j) cm = fmaxf(cm, __uint_as_float(r[j]));
+            if (cm > m) {
+                const float f = ex2_approx((m - cm) * kLog2e);
+                s0 *= f;
+                s1 *= f;
+                m = cm;
+            }
+            const float nm = -m * kLog2e;
+#pragma unroll
+            for (int j = 0; j < 32; j += 2) {
+                s0 += ex2_approx(fmaf(__uint_as_float(r[j]), kLog2e, nm));
+                s1 += ex2_approx(fmaf(__uint_as_float(r[j + 1]), kLog2e, nm));
+            }
+            if ((ycol >> 5) == c && ycol >= 0) {
+                const int jj = ycol & 31;
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                    if (j == jj) zyv = __uint_as_float(r[j]);
+            }
+        }
+        if (row < p.T) {
+            const size_t o = (size_t)(n0 / BN) * (size_t)p.T + (size_t)row;
+            p.part_m[o] = m;
+            p.part_s[o] = s0 + s1;
+            if (ycol >= 0 && ycol < ncols) p.zy[row] = zyv;
+        }
+    }
+    __device__ void finish() {}
+};
+
+// per-tile pairs -> lse, log pi(y), row state; one thread per row
+__global__ void __launch_bounds__(256)
+head_merge_kernel(int64_t T, int vocab, int n_tiles, const float* __restrict__ part_m,
+                  const float* __restrict__ part_s, const float* __restrict__ zy,
+                  const int32_t* __restrict__ targets, const uint8_t* __restrict__ mask, Workspace ws) {
+    const int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= T) return;
+    const bool on = mask ? (mask[r] != 0) : true;
+    const int32_t y = targets[r];
+    if (!on || y < 0 || y >= vocab) {
+        ws.row_state[r] = on ? ROW_BAD_TOKEN : ROW_MASKED;
+        ws.lse[r] = 0.0;
+        ws.token_logp[r] = 0.0;
+        ws.row_max[r] = 0.f;
+        return;
+    }
+    float M = -INFINITY;
+    for (int j = 0; j < n_tiles; ++j) M = fmaxf(M, part_m[(size_t)j * T + r]);
+    double S = 0.0;
+    for (int j = 0; j < n_tiles; ++j) {
+        const size_t o = (size_t)j * T + r;
+        S += (double)part_s[o] * exp((double)part_m[o] - (double)M);
+    }
+    const double lse = (double)M + log(S);
+    ws.lse[r] = lse;
+    ws.token_logp[r] = (double)zy[r] - lse;
+    ws.row_max[r] = M;
+    ws.row_state[r] = ROW_OK;
+}
+
+// ---- stores through shared memory and TMA -----------------------------------------------------------
+
+// A warp hands 32 rows x 128 bytes (its 32 accumulator lanes x 64 bf16 or 32 floats) to one tiled
+// TMA store.  Two 4 KB buffers alternate; a buffer is rewritten only after the store issued two
+// steps earlier has finished reading it.  Stores are clipped at the matrix bounds by the TMA unit.
+struct WarpStore {
+    uint8_t* stage;
+    int lane;
+    uint32_t n;  // stores issued
+    __device__ WarpStore(uint8_t* s, int l) : stage(s), lane(l), n(0) {}
+    __device__ uint8_t* begin() {
+        if (n >= 2) {
+            if (lane == 0) bulk_wait_read<1>();
+            __syncwarp();
+        }
+        return stage + (n & 1u) * 4096u;
+    }
+    __device__ void commit(const CUtensorMap* map, uint8_t* buf, int x, int y) {
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+            tma_store_2d(map, buf, x, y);
+            bulk_commit();
+        }
+        ++n;
+    }
+    __device__ void finish() {
+        if (lane == 0) bulk_wait_all<0>();
+        __syncwarp();
+    }
+};
+
+// ---- backward epilogue 1: dz in bf16 -------------------------------------------------------------------
+
+struct DzStore {
+    struct Params {
+        CUtensorMap map;  // dz [T, V] bf16, box 64 x 32
+        const double* lse;
+        const double* coef;
+        const double* coef_log2;
+        const uint8_t* row_state;
+        const int32_t* targets;
+        int T, V, seq_len;
+    };
+    const Params& p;
+    const int quarter, lane;
+    WarpStore st;
+    __device__ DzStore(const Params& p_, uint8_t* stage, int q, int l) : p(p_), quarter(q), lane(l), st(stage, l) {}
+
+    __device__ void tile(int m0, int n0, uint32_t taddr) {
+        const int row = m0 + quarter * 32 + lane;
+        const int ncols = min(BN, p.V - n0);
+        float c = -INFINITY, g = 0.f;  // dead row: 2^-inf = 0 everywhere, nothing subtracted
+        uint32_t sign2 = 0;
+        int ycol = -1;
+        if (row < p.T && p.row_state[row] == ROW_OK) {
+            const int n = row / p.seq_len;
+            const double gd = p.coef[n];
+            if (gd != 0.0) {
+                c = (float)fma(-p.lse[row], kLog2eD, p.coef_log2[n]);
+                g = (float)gd;
+                sign2 = (gd < 0.0) ? 0x80008000u : 0u;
+                ycol = p.targets[row] - n0;
+            }
+        }
+#pragma unroll 1
+        for (int q = 0; q * 64 < ncols; ++q) {
+            uint8_t* buf = st.begin();
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const int cc = q * 2 + half;
+                uint32_t r[32];
+                tmem_ld32(taddr + cc * 32, r);
+                tmem_ld_wait();
+                uint32_t o[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const float lo = ex2_approx(fmaf(__uint_as_float(r[2 * j]), kLog2e, c));
+                    const float hi = ex2_approx(fmaf(__uint_as_float(r[2 * j + 1]), kLog2e, c));
+                    o[j] = pack_bf16x2(lo, hi) ^ sign2;
+                }
+                if (ycol >= 0 && (ycol >> 5) == cc) {  // the sampled token: g (p_y - 1), formed in float
+                    const int jj = ycol & 31;
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        if (j == (jj >> 1)) {
+                            const float lo = ex2_approx(fmaf(__uint_as_float(r[2 * j]), kLog2e, c));
+                            const float hi = ex2_approx(fmaf(__uint_as_float(r[2 * j + 1]), kLog2e, c));
+                            float vlo = (g < 0.f) ? -lo : lo, vhi = (g < 0.f) ? -hi : hi;
+                            if (jj & 1) vhi -= g; else vlo -= g;
+                            o[j] = pack_bf16x2(vlo, vhi);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    *reinterpret_cast<uint4*>(buf + swz128(lane, half * 4 + k)) =
+                        make_uint4(o[4 * k], o[4 * k + 1], o[4 * k + 2], o[4 * k + 3]);
+            }
+            st.commit(&p.map, buf, n0 + q * 64, m0 + quarter * 32);
+        }
+    }
+    __device__ void finish() { st.finish(); }
+};
+
+// ---- backward epilogues 2 and 3: plain stores ------------------------------------------------------------
+
+struct StoreBf16 {  // dh
+    struct Params {
+        CUtensorMap map;  // [M, N] bf16, box 64 x 32
+        int N;
+    };
+    const Params& p;
+    const int quarter, lane;
+    WarpStore st;
+    __device__ StoreBf16(const Params& p_, uint8_t* stage, int q, int l) : p(p_), quarter(q), lane(l), st(stage, l) {}
+    __device__ void tile(int m0, int n0, uint32_t taddr) {
+        const int ncols = min(BN, p.N - n0);
+#pragma unroll 1
+        for (int q = 0; q * 64 < ncols; ++q) {
+            uint8_t* buf = st.begin();
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                uint32_t r[32];
+                tmem_ld32(taddr + (q * 2 + half) * 32, r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    uint32_t o[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        o[j] = pack_bf16x2(__uint_as_float(r[8 * k + 2 * j]), __uint_as_float(r[8 * k + 2 * j + 1]));
+                    *reinterpret_cast<uint4*>(buf + swz128(lane, half * 4 + k)) = make_uint4(o[0], o[1], o[2], o[3]);
+                }
+            }
+            st.commit(&p.map, buf, n0 + q * 64, m0 + quarter * 32);
+        }
+    }
+    __device__ void finish() { st.finish(); }
+};
+
+struct StoreF32 {  // dW
+    struct Params {
+        CUtensorMap map;  // [M, N] float, box 32 x 32
+        int N;
+    };
+    const Params& p;
+    const int quarter, lane;
+    WarpStore st;
+    __device__ StoreF32(const Params& p_, uint8_t* stage, int q, int l) : p(p_), quarter(q), lane(l), st(stage, l) {}
+    __device__ void tile(int m0, int n0, uint32_t taddr) {
+        const int ncols = min(BN, p.N - n0);
+#pragma unroll 1
+        for (int c = 0; c * 32 < ncols; ++c) {
+            uint8_t* buf = st.begin();
+            uint32_t r[32];
+            tmem_ld32(taddr + c * 32, r);
+            tmem_ld_wait();
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                *reinterpret_cast<uint4*>(buf + swz128(lane, k)) =
+                    make_uint4(r[4 * k], r[4 * k + 1], r[4 * k + 2], r[4 * k + 3]);
+            st.commit(&p.map, buf, n0 + c * 32, m0 + quarter * 32);
+        }
+    }
+    __device__ void finish() { st.finish(); }
+};
+
+__global__ void clear_status_kernel(int* status) { *status = 0; }
+
+// the status word of the scratch -> the statistics block(s), after everything else
+__global__ void publish_status_kernel(const int* status, rapid_stats_t* a, rapid_stats_t* b) {
+    if (*status != 0) {
+        if (a) atomicMax(&a->status, *status);
+        if (b) atomicMax(&b->status, *status);
+    }
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+rapid_status_t check_head_args(const rapid_desc_t* d, int32_t D) {
+    if (!d) return RAPID_ERR_INVALID_ARG;
+    if (d->n_seq <= 0 || d->n_groups <= 0 || d->seq_len <= 0 || d->vocab <= 0 || D <= 0) return RAPID_ERR_INVALID_ARG;
+    if (!(d->eta > 0.0)) return RAPID_ERR_INVALID_ARG;
+    if (d->dtype != RAPID_BF16) return RAPID_ERR_INVALID_ARG;
+    if (d->ld < d->vocab) return RAPID_ERR_INVALID_ARG;
+    if (d->flags & RAPID_FLAG_ADV_INPUT_IS_WEIGHT) return RAPID_ERR_INVALID_ARG;
+    if (d->ld % 8 != 0 || D % 8 != 0) return RAPID_ERR_ALIGNMENT;  // 16-byte row pitches for TMA
+    return RAPID_OK;
+}
+
+}  // namespace
+
+}  // namespace rapid
+
+using namespace rapid;
+using namespace rapid::umma;
+
+extern "C" rapid_status_t rapid_fused_head_workspace_bytes(const rapid_desc_t* desc, int32_t hidden_dim,
+                                                           size_t* bytes) {
+    if (!bytes) return RAPID_ERR_INVALID_ARG;
+    rapid_status_t s = check_head_args(desc, hidden_dim);
+    if (s != RAPID_OK) return s;
+    const size_t base = align_up(carve_workspace(*desc, nullptr, nullptr), 1024);
+    *bytes = carve_head(*desc, nullptr, base, nullptr);
+    return RAPID_OK;
+}
+
+extern "C" rapid_status_t rapid_pg_loss_fused_head(
+    const rapid_desc_t* desc, int32_t hidden_dim, const void* hidden, const void* w_vocab,
+    const int32_t* targets, const uint8_t* mask, const float* behav_logp, const float* rewards,
+    const int32_t* group_offsets, float* loss, void* dhidden, void* dW, float* token_logp, float* adv,
+    rapid_stats_t* stats, void* workspace, size_t workspace_bytes, void* stream) {
+    rapid_status_t s = check_head_args(desc, hidden_dim);
+    if (s != RAPID_OK) return s;
+    if (!hidden || !w_vocab || !targets || !behav_logp || !rewards || !group_offsets || !loss || !dhidden || !dW)
+        return RAPID_ERR_INVALID_ARG;
+    if (!aligned16(hidden) || !aligned16(w_vocab) || !aligned16(dhidden) || !aligned16(dW)) return RAPID_ERR_ALIGNMENT;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) % 1024) != 0) return RAPID_ERR_WORKSPACE;
+    Workspace ws;
+    HeadScratch hs;
+    const size_t base = align_up(carve_workspace(*desc, workspace, &ws), 1024);
+    const size_t need = carve_head(*desc, workspace, base, &hs);
+    if (workspace_bytes < need) return RAPID_ERR_WORKSPACE;
+
+    int dev = 0, major = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return RAPID_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return RAPID_ERR_CUDA;
+    if (major != 10) return RAPID_ERR_UNSUPPORTED;
+
+    const int64_t T = (int64_t)desc->n_seq * desc->seq_len;
+    const int V = desc->vocab, D = hidden_dim;
+    const int64_t ld = desc->ld;
+    if (T > 0x7fffffff) return RAPID_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+    // tensor maps (host structs, passed to the kernels by value)
+    CUtensorMap h_k, w_mn, w_k, h_mn, dz_k, dz_mn;
+    DzStore::Params dzp;
+    StoreBf16::Params dhp;
+    StoreF32::Params dwp;
+    bool ok = make_map_bf16(&h_k, hidden, T, D, D, BK, BM)              // A of forward: rows x K
+              && make_map_bf16(&w_mn, w_vocab, D, V, ld, 64, BK)        // B of forward: K x N
+              && make_map_bf16(&w_k, w_vocab, D, V, ld, BK, BN)         // B of dh: N(=D) x K(=V)
+              && make_map_bf16(&h_mn, hidden, T, D, D, 64, BK)          // A of dW: K(=T) x M(=D)
+              && make_map_bf16(&dz_k, hs.dz, T, V, hs.ldz, BK, BM)      // A of dh: rows x K(=V)
+              && make_map_bf16(&dz_mn, hs.dz, T, V, hs.ldz, 64, BK)     // B of dW: K(=T) x N(=V)
+              && make_map_bf16(&dzp.map, hs.dz, T, V, hs.ldz, 64, 32)   // stores
+              && make_map_bf16(&dhp.map, dhidden, T, D, D, 64, 32) &&
+              make_map_f32(&dwp.map, dW, D, V, ld, 32, 32);
+    if (!ok) return RAPID_ERR_CUDA;
+
+    const int mT = (int)((T + BM - 1) / BM), nV = (V + BN - 1) / BN;
+    clear_status_kernel<<<1, 1, 0, st>>>(hs.status);
+
+    // forward
+    FwdStats::Params fp{hs.part_m, hs.part_s, hs.zy, targets, (int)T, V};
+    Shape fwd{mT, nV, (D + BK - 1) / BK, M_FASTEST};
+    if (launch_gemm<FwdStats, false, true>(h_k, w_mn, fwd, sms, hs.status, fp, st) != cudaSuccess) return RAPID_ERR_CUDA;
+    head_merge_kernel<<<(unsigned)((T + 255) / 256), 256, 0, st>>>(T, V, hs.n_tiles, hs.part_m, hs.part_s, hs.zy,
+                                                                   targets, mask, ws);
+    if (cudaGetLastError() != cudaSuccess) return RAPID_ERR_CUDA;
+    if (launch_seq_reduce(*desc, behav_logp, token_logp, ws, st) != cudaSuccess) return RAPID_ERR_CUDA;
+    if (launch_finalize(*desc, rewards, group_offsets, loss, adv, stats, ws, st) != cudaSuccess) return RAPID_ERR_CUDA;
+
+    // backward: dz, then dh and dW
+    dzp.lse = ws.lse;
+    dzp.coef = ws.coef;
+    dzp.coef_log2 = ws.coef_log2;
+    dzp.row_state = ws.row_state;
+    dzp.targets = targets;
+    dzp.T = (int)T;
+    dzp.V = V;
+    dzp.seq_len = desc->seq_len;
+    if (launch_gemm<DzStore, false, true>(h_k, w_mn, fwd, sms, hs.status, dzp, st) != cudaSuccess) return RAPID_ERR_CUDA;
+
+    dhp.N = D;
+    Shape sdh{mT, (D + BN - 1) / BN, (V + BK - 1) / BK, N_FASTEST};
+    if (launch_gemm<StoreBf16, false, false>(dz_k, w_k, sdh, sms, hs.status, dhp, st) != cudaSuccess) return RAPID_ERR_CUDA;
+
+    dwp.N = V;
+    Shape sdw{(D + BM - 1) / BM, nV, (int)((T + BK - 1) / BK), M_FASTEST};
+    if (launch_gemm<StoreF32, true, true>(h_mn, dz_mn, sdw, sms, hs.status, dwp, st) != cudaSuccess) return RAPID_ERR_CUDA;
+
+    publish_status_kernel<<<1, 1, 0, st>>>(hs.status, stats, ws.stats);
+    return cudaGetLastError() == cudaSuccess ? RAPID_OK : RAPID_ERR_CUDA;
+}

@@ -38,7 +38,8 @@ constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kThreads = 192;
 constexpr int kEpiThreads = 128;
 constexpr int kTmemCols = 512;
-constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 1024;  // + slack to align to 1024
+constexpr int kEpiStageBytes = 8192;  // per epilogue warp: two 4 KB buffers for outgoing TMA stores
+constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 4 * kEpiStageBytes + 1024;  // + slack to align to 1024
 
 enum TileOrder : int { M_FASTEST = 0, N_FASTEST = 1 };
 
@@ -103,6 +104,20 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// shared -> global tiled store of one box (clipped at the tensor's bounds), tracked by the issuing
+// thread's bulk group.  x * element size must be a multiple of 16 bytes and never negative.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void* smem_src, int x, int y) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(map),
+                 "r"(smem_u32(smem_src)), "r"(x), "r"(y)
+                 : "memory");
+}
+
+// Byte offset, inside a 128-byte-swizzled box whose rows are 128 bytes, of 16-byte chunk `chunk`
+// (0..7) of row `row`: the chunk index is XORed with the row index modulo 8.
+__device__ __forceinline__ uint32_t swz128(int row, int chunk) {
+    return (uint32_t)row * 128u + (uint32_t)((chunk ^ (row & 7)) << 4);
+}
+
 // ---- descriptors -----------------------------------------------------------------------------------
 
 // Shared-memory operand descriptor, 128-byte swizzle.  Fields (bit positions): start address >> 4
@@ -133,15 +148,20 @@ __host__ __device__ constexpr uint32_t instr_desc(bool a_mn, bool b_mn) {
 // ---- the kernel ------------------------------------------------------------------------------------
 
 // Epi must provide:
-//   struct Params;                                    (trivially copyable)
-//   __device__ static void tile(const Params&, int m0, int n0, int row_in_tile, uint32_t taddr);
-// `taddr` addresses lane `row_in_tile & ~31` (this warp's 32 lanes), column 0 of the tile's
-// accumulator; the functor reads it with tmem_ld32(taddr + column, ...) and MUST end with
-// tmem_ld_wait().  All 32 lanes of the warp call it together.
+//   struct Params;                                    (trivially copyable; passed __grid_constant__, so
+//                                                      a CUtensorMap member may be handed to TMA)
+//   __device__ Epi(const Params&, uint8_t* stage, int quarter, int lane);
+//   __device__ void tile(int m0, int n0, uint32_t taddr);
+//   __device__ void finish();
+// One object lives per epilogue warp for the whole kernel.  `stage` is that warp's kEpiStageBytes
+// of shared memory (1024-byte aligned).  `taddr` addresses this warp's 32 accumulator lanes
+// (rows m0 + 32 * quarter + lane), column 0 of the tile; the functor reads it with
+// tmem_ld32(taddr + column, ...) and every load must have been waited for (tmem_ld_wait) before
+// tile() returns.  All 32 lanes call tile() and finish() together.
 template <class Epi, bool A_MN, bool B_MN>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, Shape shape,
-            int* status, typename Epi::Params ep) {
+            int* status, const __grid_constant__ typename Epi::Params ep) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     __shared__ __align__(8) uint64_t full_bar[kStages];
@@ -282,7 +302,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     } else {
         // ------------------------------------ epilogue ------------------------------------------------
         const int quarter = warp & 3;  // the 32 accumulator lanes this warp may read
-        const int row_in_tile = quarter * 32 + lane;
+        Epi epi(ep, smem + (size_t)kStages * kStageBytes + (size_t)(warp - 2) * kEpiStageBytes, quarter, lane);
         uint32_t tile_iter = 0;
         for (int idx = blockIdx.x; idx < total; idx += gridDim.x, ++tile_iter) {
             int mb, nb;
@@ -293,11 +313,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             if (!__all_sync(0xffffffffu, got)) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
-            Epi::tile(ep, mb * BM, nb * BN, row_in_tile, taddr);
+            epi.tile(mb * BM, nb * BN, taddr);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&tempty_bar[acc]);
         }
+        __syncwarp();
+        epi.finish();
     }
     __syncthreads();
     if (warp == 1) {
@@ -315,6 +337,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 // rejects the arguments.
 bool make_map_bf16(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint64_t ld,
                    uint32_t box_cols, uint32_t box_rows);
+// The same for a float matrix (ld * 4 bytes a multiple of 16; box_cols * 4 = 128 bytes).
+bool make_map_f32(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint64_t ld,
+                  uint32_t box_cols, uint32_t box_rows);
 
 template <class Epi, bool A_MN, bool B_MN>
 cudaError_t launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const Shape& shape, int sm_count,
