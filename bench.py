@@ -50,6 +50,16 @@ def load_peaks():
     return 6650.0, "fallback"
 
 
+def load_tensor_peaks():
+    """(burst, sustained) dense bf16 TFLOP/s and where they come from."""
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            j = json.load(f)
+        return float(j["bf16_tflops"]), float(j.get("bf16_tflops_sustained", j["bf16_tflops"])), "measured"
+    return 1590.0, 1400.0, "fallback"
+
+
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons for one GPU while the timed region runs."""
 
@@ -346,6 +356,148 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------------------------
+# the fused LM-head form (--workload fused): hidden states and the LM-head weight in, no logits
+# ------------------------------------------------------------------------------------------------
+
+def run_fused(args):
+    from paper_2510_03515_b200 import binding as rb
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    rb.lib()
+    w = synth.CONFIGS["fused"].scaled(seed=synth.CONFIGS["fused"].seed + 1000 * rank)
+    if args.seq_len:
+        w = w.scaled(seq_len=args.seq_len)
+    b = synth.make_head(w, device=dev)
+    T, V, D, N = w.n_rows, w.vocab, w.hidden, w.n_seq
+    desc = rb.make_desc(N, w.seq_len, V, w.n_prompts, torch.bfloat16, V, 2.0, 0)
+    ws = rb.alloc_fused_head_workspace(desc, D, dev)
+    loss = torch.zeros(1, device=dev)
+    dh = torch.empty((T, D), dtype=torch.bfloat16, device=dev)
+    dW = torch.empty((D, V), dtype=torch.float32, device=dev)
+    tl = torch.empty(T, device=dev)
+    adv = torch.empty(N, device=dev)
+    stats = rb.alloc_stats(dev)
+    behav = torch.full((T,), -12.0, device=dev)
+
+    def step(hid=None, wv=None, bh=None):
+        rb.rapid_pg_loss_fused_head(desc, b["hidden"] if hid is None else hid, b["w_vocab"] if wv is None else wv,
+                                    b["targets"], b["mask"], behav if bh is None else bh, b["rewards"],
+                                    b["group_offsets"], loss, dh, dW, tl, adv, stats, ws)
+
+    step()   # the library's own token log-probs seed the synthetic behaviour log-probs (input synthesis)
+    torch.cuda.synchronize()
+    behav = (tl + b["behav_noise"]).contiguous()
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    if dist:
+        dist.barrier()
+    torch.cuda.synchronize()
+    if sampler:
+        sampler.start()
+        time.sleep(0.25)
+    t0w = time.time()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for _ in range(args.steps):
+        step()
+    end.record()
+    torch.cuda.synchronize()
+    t1w = time.time()
+    if dist:
+        dist.barrier()
+    clocks = sampler.stop(t0w, t1w) if sampler else None
+    ms = start.elapsed_time(end)
+    n_tokens = int(b["mask"].sum().item())
+    tokens = float(n_tokens)
+    if dist:
+        t = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+        tk = torch.tensor([tokens], device=dev, dtype=torch.float64)
+        dist.all_reduce(tk, op=dist.ReduceOp.SUM)
+        tokens = float(tk.item())
+    ms_per_step = ms / args.steps
+    st = rb.read_stats(stats)
+
+    # end to end: hidden states, weight and per-token arrays start in pinned host memory
+    e2e = None
+    if not args.skip_e2e:
+        names = ("hidden", "w_vocab")
+        host = {k: b[k].cpu().pin_memory() for k in names}
+        h_behav = behav.cpu().pin_memory()
+        d_in = {k: torch.empty_like(b[k]) for k in names}
+        d_behav = torch.empty_like(behav)
+        h_loss = torch.empty(1, dtype=torch.float32).pin_memory()
+        h2d = sum(v.numel() * v.element_size() for v in host.values()) + h_behav.numel() * 4
+
+        def e2e_step():
+            for k in names:
+                d_in[k].copy_(host[k], non_blocking=True)
+            d_behav.copy_(h_behav, non_blocking=True)
+            step(d_in["hidden"], d_in["w_vocab"], d_behav)
+            h_loss.copy_(loss, non_blocking=True)
+            torch.cuda.current_stream().synchronize()
+
+        e2e_step()
+        if dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+        k = max(1, min(args.e2e_steps, args.steps))
+        s2, e2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s2.record()
+        for _ in range(k):
+            e2e_step()
+        e2.record()
+        torch.cuda.synchronize()
+        ems = s2.elapsed_time(e2)
+        if dist:
+            t = torch.tensor([ems], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ems = float(t.item())
+        e2e = {"value": tokens * k / (ems * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+               "d2h_bytes_per_step": 4, "steps": k, "ms_per_step": ems / k}
+    if rank != 0:
+        if dist:
+            dist.destroy_process_group()
+        return
+    burst, sustained, kind = load_tensor_peaks()
+    flops = 4 * 2.0 * T * D * V   # forward, recompute, dhidden, dW
+    ach = flops / (ms_per_step * 1e-3) / 1e12
+    line = {
+        "metric": "fused LM-head PG loss fwd+bwd tokens/sec at V=151936 bf16", "value": tokens / (ms_per_step * 1e-3),
+        "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "fused", "prompts": w.n_prompts, "generations_per_prompt": w.group_size,
+                   "padded_len": w.seq_len, "rows_per_gpu": T, "hidden": D, "vocab": V,
+                   "l2_policy": "inputs larger than L2 (0.47 GB weight, 5 GB dlogits scratch per step)",
+                   "eta": 2.0, "parallelism": f"dp{world} (by prompt group, no data-path collective)"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": 9 * args.steps,
+        "roofline": {"bound": "tensor", "kernel": "umma gemm_kernel x4 (forward statistics, dlogits, dhidden, dW)",
+                     "achieved": ach, "peak": sustained, "peak_kind": kind + " sustained", "unit": "TFLOP/s",
+                     "frac": ach / sustained, "frac_of_burst": ach / burst, "flops_per_step": flops,
+                     "traffic": None},
+        "cpu_baseline": None,
+        "stats": {"n_clipped": st["n_clipped"], "mean_log_cw": st["mean_log_cw"], "loss": st["loss"],
+                  "status": st["status"]},
+    }
+    print(json.dumps(line), flush=True)
+    if dist:
+        dist.destroy_process_group()
+
+
 # DRAM traffic of pass 2 per algorithmic byte, from the ncu capture summarised under profiles/
 # (dram__bytes_read.sum + dram__bytes_write.sum of a smaller launch, which scales with rows).
 TRAFFIC_P2_PER_BYTE = None
@@ -430,6 +582,8 @@ def main():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="slm", choices=["slm", "fused"],
+                    help="slm: the logits-in path the metric is quoted on (default); fused: the LM-head form")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--skip-e2e", action="store_true", help="leave out the host-buffer leg (profiling)")
     ap.add_argument("--skip-cpu", action="store_true", help="leave out the CPU oracle timing (profiling)")
@@ -440,7 +594,10 @@ def main():
         run_reference(args)
     else:
         args.warmup = max(args.warmup, 3)
-        run_ours(args)
+        if args.workload == "fused":
+            run_fused(args)
+        else:
+            run_ours(args)
 
 
 if __name__ == "__main__":
