@@ -118,13 +118,33 @@ struct FwdStats {
     __device__ void finish() {}
 };
 
-// per-tile pairs -> lse, log pi(y), row state; one thread per row
-__global__ void __launch_bounds__(256)
+// per-tile pairs -> lse, log pi(y), row state.  A CTA covers 32 rows; its 8 warps each take every
+// 8th tile (loads are coalesced across the 32 rows), and the partial (max, sum) pairs are combined
+// through shared memory in double.
+constexpr int kMergeRows = 32;
+constexpr int kMergeSlices = 8;
+
+__global__ void __launch_bounds__(kMergeRows * kMergeSlices)
 head_merge_kernel(int64_t T, int vocab, int n_tiles, const float* __restrict__ part_m,
                   const float* __restrict__ part_s, const float* __restrict__ zy,
                   const int32_t* __restrict__ targets, const uint8_t* __restrict__ mask, Workspace ws) {
-    const int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (r >= T) return;
+    __shared__ float sh_m[kMergeSlices][kMergeRows];
+    __shared__ double sh_s[kMergeSlices][kMergeRows];
+    const int lane = threadIdx.x & 31, slice = threadIdx.x >> 5;
+    const int64_t r = (int64_t)blockIdx.x * kMergeRows + lane;
+    float M = -INFINITY;
+    double S = 0.0;
+    if (r < T) {
+        for (int j = slice; j < n_tiles; j += kMergeSlices) M = fmaxf(M, part_m[(size_t)j * T + r]);
+        for (int j = slice; j < n_tiles; j += kMergeSlices) {
+            const size_t o = (size_t)j * T + r;
+            S += (double)part_s[o] * exp((double)part_m[o] - (double)M);
+        }
+    }
+    sh_m[slice][lane] = M;
+    sh_s[slice][lane] = S;
+    __syncthreads();
+    if (slice != 0 || r >= T) return;
     const bool on = mask ? (mask[r] != 0) : true;
     const int32_t y = targets[r];
     if (!on || y < 0 || y >= vocab) {
@@ -134,17 +154,15 @@ head_merge_kernel(int64_t T, int vocab, int n_tiles, const float* __restrict__ p
         ws.row_max[r] = 0.f;
         return;
     }
-    float M = -INFINITY;
-    for (int j = 0; j < n_tiles; ++j) M = fmaxf(M, part_m[(size_t)j * T + r]);
-    double S = 0.0;
-    for (int j = 0; j < n_tiles; ++j) {
-        const size_t o = (size_t)j * T + r;
-        S += (double)part_s[o] * exp((double)part_m[o] - (double)M);
-    }
-    const double lse = (double)M + log(S);
+    float Mr = sh_m[0][lane];
+    for (int k = 1; k < kMergeSlices; ++k) Mr = fmaxf(Mr, sh_m[k][lane]);
+    double Sr = 0.0;
+    for (int k = 0; k < kMergeSlices; ++k)
+        if (sh_s[k][lane] > 0.0) Sr += sh_s[k][lane] * exp((double)sh_m[k][lane] - (double)Mr);
+    const double lse = (double)Mr + log(Sr);
     ws.lse[r] = lse;
     ws.token_logp[r] = (double)zy[r] - lse;
-    ws.row_max[r] = M;
+    ws.row_max[r] = Mr;
     ws.row_state[r] = ROW_OK;
 }
 
@@ -409,8 +427,8 @@ extern "C" rapid_status_t rapid_pg_loss_fused_head(
     FwdStats::Params fp{hs.part_m, hs.part_s, hs.zy, targets, (int)T, V};
     Shape fwd{mT, nV, (D + BK - 1) / BK, M_FASTEST};
     if (launch_gemm<FwdStats, false, true>(h_k, w_mn, fwd, sms, hs.status, fp, st) != cudaSuccess) return RAPID_ERR_CUDA;
-    head_merge_kernel<<<(unsigned)((T + 255) / 256), 256, 0, st>>>(T, V, hs.n_tiles, hs.part_m, hs.part_s, hs.zy,
-                                                                   targets, mask, ws);
+    head_merge_kernel<<<(unsigned)((T + kMergeRows - 1) / kMergeRows), kMergeRows * kMergeSlices, 0, st>>>(
+        T, V, hs.n_tiles, hs.part_m, hs.part_s, hs.zy, targets, mask, ws);
     if (cudaGetLastError() != cudaSuccess) return RAPID_ERR_CUDA;
     if (launch_seq_reduce(*desc, behav_logp, token_logp, ws, st) != cudaSuccess) return RAPID_ERR_CUDA;
     if (launch_finalize(*desc, rewards, group_offsets, loss, adv, stats, ws, st) != cudaSuccess) return RAPID_ERR_CUDA;
