@@ -74,10 +74,15 @@ enum {
      * shown after Eq. 4, which the paper states but does not use).                              */
     RAPID_FLAG_LEAVE_ONE_OUT = 8u,
     /* With LEAVE_ONE_OUT: divide by N_k, as that display is printed.                            */
-    RAPID_FLAG_LOO_LITERAL_DIVISOR = 16u
+    RAPID_FLAG_LOO_LITERAL_DIVISOR = 16u,
+    /* The normaliser Z of Eq. 3 is desc->norm_z instead of being counted from this call's own    */
+    /* generations (or tokens).  For a mini-batch whose prompt groups are spread over several     */
+    /* GPUs: every rank passes the global N (or the global token count), so that the per-rank     */
+    /* losses and gradients simply add up to those of the whole mini-batch.                       */
+    RAPID_FLAG_NORM_GIVEN = 32u
 };
 
-/* Problem descriptor (host memory, plain data, 40 bytes). */
+/* Problem descriptor (host memory, plain data, 48 bytes). */
 typedef struct rapid_desc {
     int32_t n_seq;    /* N: generations in the mini-batch (N_step in the paper)                   */
     int32_t seq_len;  /* L: padded response length; rows T = N * L                                */
@@ -87,6 +92,7 @@ typedef struct rapid_desc {
     int32_t dtype;    /* rapid_dtype_t of logits and dlogits                                      */
     uint32_t flags;   /* RAPID_FLAG_* bits                                                        */
     double eta;       /* importance-weight cap of Eq. 5; +inf gives Eq. 4; must be > 0            */
+    double norm_z;    /* Z of Eq. 3 when RAPID_FLAG_NORM_GIVEN is set (> 0, finite); else ignored  */
 } rapid_desc_t;
 
 /* Side statistics (DEVICE memory, written by the finalize step, 48 bytes). */

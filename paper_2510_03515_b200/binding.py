@@ -33,6 +33,7 @@ FLAG_NORM_TOKENS = 2
 FLAG_ADV_INPUT_IS_WEIGHT = 4
 FLAG_LEAVE_ONE_OUT = 8
 FLAG_LOO_LITERAL_DIVISOR = 16
+FLAG_NORM_GIVEN = 32
 
 # every symbol declared in include/rapid_pg.h
 EXPORTS = (
@@ -45,7 +46,7 @@ EXPORTS = (
 class RapidDesc(C.Structure):
     _fields_ = [("n_seq", C.c_int32), ("seq_len", C.c_int32), ("vocab", C.c_int32),
                 ("n_groups", C.c_int32), ("ld", C.c_int64), ("dtype", C.c_int32),
-                ("flags", C.c_uint32), ("eta", C.c_double)]
+                ("flags", C.c_uint32), ("eta", C.c_double), ("norm_z", C.c_double)]
 
 
 class RapidStats(C.Structure):
@@ -124,7 +125,8 @@ def _check(code: int, where: str) -> None:
 
 
 def make_desc(n_seq: int, seq_len: int, vocab: int, n_groups: int, dtype: torch.dtype,
-              ld: Optional[int] = None, eta: float = 2.0, flags: int = 0) -> RapidDesc:
+              ld: Optional[int] = None, eta: float = 2.0, flags: int = 0,
+              norm_z: float = 0.0) -> RapidDesc:
     if dtype == torch.float32:
         dt = RAPID_F32
     elif dtype == torch.bfloat16:
@@ -132,7 +134,7 @@ def make_desc(n_seq: int, seq_len: int, vocab: int, n_groups: int, dtype: torch.
     else:
         raise TypeError("logits must be float32 or bfloat16")
     return RapidDesc(n_seq, seq_len, vocab, n_groups, vocab if ld is None else ld, dt, flags,
-                     float(eta))
+                     float(eta), float(norm_z))
 
 
 def rapid_workspace_bytes(desc: RapidDesc) -> int:
@@ -263,12 +265,12 @@ class PgResult:
 
 def pg_loss(logits: torch.Tensor, targets, mask, behav_logp, rewards, group_offsets, n_seq: int,
             seq_len: int, eta: float = 2.0, flags: int = 0, in_place: bool = False,
-            workspace: Optional[torch.Tensor] = None) -> PgResult:
+            workspace: Optional[torch.Tensor] = None, norm_z: float = 0.0) -> PgResult:
     """Convenience wrapper: allocate the outputs and make ONE rapid_pg_loss_fwd_bwd call."""
     T, ld = logits.shape[0], logits.stride(0)
     vocab = logits.shape[1]
     assert T == n_seq * seq_len
-    desc = make_desc(n_seq, seq_len, vocab, group_offsets.numel() - 1, logits.dtype, ld, eta, flags)
+    desc = make_desc(n_seq, seq_len, vocab, group_offsets.numel() - 1, logits.dtype, ld, eta, flags, norm_z)
     dev = logits.device
     ws = workspace if workspace is not None else alloc_workspace(desc, dev)
     dlogits = logits if in_place else torch.empty_like(logits)

@@ -17,6 +17,7 @@ rapid_status_t check_desc_basic(const rapid_desc_t* d) {
     if (!d) return RAPID_ERR_INVALID_ARG;
     if (d->n_seq <= 0 || d->n_groups <= 0) return RAPID_ERR_INVALID_ARG;
     if (!(d->eta > 0.0)) return RAPID_ERR_INVALID_ARG;  // also rejects NaN
+    if ((d->flags & RAPID_FLAG_NORM_GIVEN) && !(d->norm_z > 0.0 && d->norm_z < INFINITY)) return RAPID_ERR_INVALID_ARG;
     return RAPID_OK;
 }
 

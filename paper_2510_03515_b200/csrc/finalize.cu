@@ -91,7 +91,7 @@ __device__ __forceinline__ T block_sum(T v, T* sh) {
 // full == false: rapid_group_advantage on caller-provided log-ratios / weights.
 template <bool full>
 __global__ void __launch_bounds__(kFinThreads)
-finalize_kernel(int n_seq, int n_groups, double eta, uint32_t flags,
+finalize_kernel(int n_seq, int n_groups, double eta, double norm_z, uint32_t flags,
                 const float* __restrict__ rewards, const double* __restrict__ slr_in,
                 const int32_t* __restrict__ group_offsets, float* __restrict__ loss_out,
                 float* __restrict__ adv_out, double* __restrict__ clipped_out,
@@ -203,7 +203,9 @@ finalize_kernel(int n_seq, int n_groups, double eta, uint32_t flags,
     }
     tokens = block_sum<long long>(tokens, sh_l);
     bad_tok = block_sum<int>(bad_tok, sh_i);
-    const double Z = (flags & RAPID_FLAG_NORM_TOKENS) ? (double)tokens : (double)n_seq;
+    const double Z = (flags & RAPID_FLAG_NORM_GIVEN)    ? norm_z
+                     : (flags & RAPID_FLAG_NORM_TOKENS) ? (double)tokens
+                                                        : (double)n_seq;
     const double log_eta = log(eta);
 
     double loss = 0.0, sum_log = 0.0, sum_abs = 0.0;
@@ -261,7 +263,7 @@ cudaError_t launch_seq_reduce(const rapid_desc_t& d, const float* behav_logp, fl
 cudaError_t launch_finalize(const rapid_desc_t& d, const float* rewards,
                             const int32_t* group_offsets, float* loss, float* adv,
                             rapid_stats_t* stats_out, const Workspace& ws, cudaStream_t stream) {
-    finalize_kernel<true><<<1, kFinThreads, 0, stream>>>(d.n_seq, d.n_groups, d.eta, d.flags, rewards,
+    finalize_kernel<true><<<1, kFinThreads, 0, stream>>>(d.n_seq, d.n_groups, d.eta, d.norm_z, d.flags, rewards,
                                                         nullptr, group_offsets, loss, adv, nullptr,
                                                         stats_out, ws);
     return cudaGetLastError();
@@ -272,7 +274,7 @@ cudaError_t launch_group_advantage(const rapid_desc_t& d, const float* rewards,
                                    float* adv, double* clipped_w, rapid_stats_t* stats_out,
                                    cudaStream_t stream) {
     Workspace none = {};
-    finalize_kernel<false><<<1, kFinThreads, 0, stream>>>(d.n_seq, d.n_groups, d.eta, d.flags,
+    finalize_kernel<false><<<1, kFinThreads, 0, stream>>>(d.n_seq, d.n_groups, d.eta, d.norm_z, d.flags,
                                                          rewards, seq_log_ratio, group_offsets,
                                                          nullptr, adv, clipped_w, stats_out, none);
     return cudaGetLastError();

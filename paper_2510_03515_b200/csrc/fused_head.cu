@@ -350,6 +350,7 @@ rapid_status_t check_head_args(const rapid_desc_t* d, int32_t D) {
     if (!d) return RAPID_ERR_INVALID_ARG;
     if (d->n_seq <= 0 || d->n_groups <= 0 || d->seq_len <= 0 || d->vocab <= 0 || D <= 0) return RAPID_ERR_INVALID_ARG;
     if (!(d->eta > 0.0)) return RAPID_ERR_INVALID_ARG;
+    if ((d->flags & RAPID_FLAG_NORM_GIVEN) && !(d->norm_z > 0.0 && d->norm_z < INFINITY)) return RAPID_ERR_INVALID_ARG;
     if (d->dtype != RAPID_BF16) return RAPID_ERR_INVALID_ARG;
     if (d->ld < d->vocab) return RAPID_ERR_INVALID_ARG;
     if (d->flags & RAPID_FLAG_ADV_INPUT_IS_WEIGHT) return RAPID_ERR_INVALID_ARG;

@@ -226,3 +226,43 @@ def test_group_advantage_zero_sum_on_device():
     R = (rng.random(512) < 0.3).astype(np.float32)
     adv, _, _ = _adv_gpu(R, None, go, 2.0, 0)
     assert np.abs(adv.reshape(64, 8).astype(np.float64).sum(1)).max() < 1e-6
+
+
+# ---- one mini-batch spread over ranks by whole prompt groups -------------------------------------------
+
+@pytest.mark.parametrize("flags", [0, rb.FLAG_NORM_TOKENS])
+def test_shards_with_given_normaliser_add_up_to_the_whole_batch(flags):
+    """Three 'ranks' (run one after another on this GPU; their kernels do not depend on each other)
+    each take whole groups and pass the global Z with RAPID_FLAG_NORM_GIVEN: losses add up to the
+    oracle's loss on the whole mini-batch and every dlogits row equals the oracle's."""
+    from paper_2510_03515_b200 import shard
+    w = synth.Workload("shards", 5, 3, 11, 1000, "bf16", 3.0, 6.0, "uniform", len_lo=3, behav_sigma=0.3,
+                       reward_mode="per_prompt", seed=29)
+    b = synth.make_batch(w)
+    L, V, N = w.seq_len, w.vocab, w.n_seq
+    bits = synth.bits_numpy(b["logits"])
+    pre = oracle.token_logp(bits, V, b["targets"].numpy(), b["mask"].numpy())
+    behav = (torch.from_numpy(pre["token_logp"]) + b["behav_noise"].double()).float()
+    full = oracle.pg_loss(bits, N, L, V, b["targets"].numpy(), b["mask"].numpy(), behav.numpy(),
+                          b["rewards"].numpy(), b["group_offsets"].numpy(), 2.0, flags, want_dlogits=True)
+    z_global = float(full["n_tokens"]) if flags & rb.FLAG_NORM_TOKENS else float(N)
+    dev = torch.device("cuda")
+    world, loss_sum, tok_sum = 3, 0.0, 0
+    for rank in range(world):
+        sh = shard.plan(b["group_offsets"].numpy(), b["lengths"].numpy(), world, rank)
+        rows = torch.from_numpy((sh.seq_index[:, None] * L + np.arange(L)[None, :]).reshape(-1))
+        res = rb.pg_loss(b["logits"][rows].contiguous().to(dev), b["targets"][rows].to(dev), b["mask"][rows].to(dev),
+                         behav[rows].to(dev), b["rewards"][torch.from_numpy(sh.seq_index)].to(dev),
+                         torch.from_numpy(sh.group_offsets).to(dev), sh.n_seq, L,
+                         flags=flags | rb.FLAG_NORM_GIVEN, norm_z=z_global)
+        torch.cuda.synchronize()
+        st = rb.read_stats(res.stats)
+        assert st["status"] == 0
+        loss_sum += st["loss"]
+        tok_sum += st["n_tokens"]
+        err = np.abs(res.dlogits.float().cpu().numpy() - full["dlogits"][rows.numpy()]).max()
+        assert err <= 4e-3
+        np.testing.assert_allclose(res.adv.cpu().numpy(), full["adv64"][sh.seq_index], rtol=0, atol=2e-4)
+    scale = max(abs(full["loss"]), 1e-3 * float(np.abs(full["coef"] * full["seq_logp"]).sum()))
+    assert abs(loss_sum - full["loss"]) / scale <= 2e-3
+    assert tok_sum == full["n_tokens"]

@@ -35,9 +35,9 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_struct_layout_matches_header():
-    assert C.sizeof(rb.RapidDesc) == 40
+    assert C.sizeof(rb.RapidDesc) == 48
     assert C.sizeof(rb.RapidStats) == 48
-    assert rb.RapidDesc.ld.offset == 16 and rb.RapidDesc.eta.offset == 32
+    assert rb.RapidDesc.ld.offset == 16 and rb.RapidDesc.eta.offset == 32 and rb.RapidDesc.norm_z.offset == 40
     assert rb.RapidStats.mean_log_cw.offset == 24
 
 
@@ -83,6 +83,8 @@ def test_argument_validation_happens_before_any_launch():
                 rb.make_desc(4, 8, 64, 0, torch.bfloat16),                 # no groups
                 rb.make_desc(4, 8, 64, 2, torch.bfloat16, eta=0.0),
                 rb.make_desc(4, 8, 64, 2, torch.bfloat16, eta=math.nan),
+                rb.make_desc(4, 8, 64, 2, torch.bfloat16, flags=rb.FLAG_NORM_GIVEN, norm_z=0.0),
+                rb.make_desc(4, 8, 64, 2, torch.bfloat16, flags=rb.FLAG_NORM_GIVEN, norm_z=math.inf),
                 rb.make_desc(4, 8, 64, 2, torch.bfloat16, flags=rb.FLAG_ADV_INPUT_IS_WEIGHT)):
         assert _call_fwd_bwd(bad) == rb.RAPID_ERR_INVALID_ARG
     odd = rb.make_desc(4, 8, 60, 2, torch.bfloat16, ld=60)                 # 120-byte pitch
