@@ -498,6 +498,105 @@ def run_fused(args):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------------------------
+# the on-policy single-pass form (--workload onpolicy): same mini-batch as slm, weights all one
+# ------------------------------------------------------------------------------------------------
+
+def run_onpolicy(args):
+    from paper_2510_03515_b200 import binding as rb
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    w = synth.CONFIGS["slm"].scaled(seed=synth.CONFIGS["slm"].seed + 1000 * rank)
+    if args.seq_len:
+        w = w.scaled(seq_len=args.seq_len, len_lo=max(1, args.seq_len // 4))
+    tok = synth.make_tokens(w)
+    T, V, N = w.n_rows, w.vocab, w.n_seq
+    logits = synth.logits_for_sequences(w, tok["targets"], 0, N, device=dev)
+    targets, mask = tok["targets"].to(dev), tok["mask"].to(dev)
+    rewards, go = tok["rewards"].to(dev), tok["group_offsets"].to(dev)
+    dlogits = torch.empty_like(logits)
+    desc = rb.make_desc(N, w.seq_len, V, w.n_prompts, logits.dtype, logits.stride(0), 2.0, 0)
+    ws = rb.alloc_workspace(desc, dev)
+    loss = torch.zeros(1, device=dev)
+    adv = torch.empty(N, device=dev)
+    stats = rb.alloc_stats(dev)
+    n_tokens = int(tok["mask"].sum().item())
+
+    def step():
+        rb.rapid_pg_loss_onpolicy_fwd_bwd(desc, logits, targets, mask, rewards, go, dlogits, loss, None, adv, stats, ws)
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    live_rows = int(((adv != 0).repeat_interleave(w.seq_len) & (mask != 0)).sum().item())
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    if dist:
+        dist.barrier()
+    torch.cuda.synchronize()
+    if sampler:
+        sampler.start()
+        time.sleep(0.25)
+    t0w = time.time()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for _ in range(args.steps):
+        step()
+    end.record()
+    torch.cuda.synchronize()
+    t1w = time.time()
+    if dist:
+        dist.barrier()
+    clocks = sampler.stop(t0w, t1w) if sampler else None
+    ms = start.elapsed_time(end)
+    tokens = float(n_tokens)
+    if dist:
+        t = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+        tk = torch.tensor([tokens], device=dev, dtype=torch.float64)
+        dist.all_reduce(tk, op=dist.ReduceOp.SUM)
+        tokens = float(tk.item())
+    if rank != 0:
+        if dist:
+            dist.destroy_process_group()
+        return
+    ms_per_step = ms / args.steps
+    st = rb.read_stats(stats)
+    peak, peak_kind = load_peaks()
+    row_bytes = V * (2 if w.dtype == "bf16" else 4)
+    algo = live_rows * 2 * row_bytes + (T - live_rows) * row_bytes   # live rows: one read + one write
+    ach = algo / (ms_per_step * 1e-3) / 1e9
+    line = {
+        "metric": "on-policy PG loss fwd+bwd tokens/sec at V=151936 bf16 (single pass)",
+        "value": tokens / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "onpolicy (slm mini-batch, mu = pi_theta)", "prompts": w.n_prompts,
+                   "generations_per_prompt": w.group_size, "padded_len": w.seq_len, "vocab": V,
+                   "logits_dtype": w.dtype, "unmasked_tokens_per_gpu": n_tokens, "live_rows_per_gpu": live_rows,
+                   "rows_per_gpu": T, "l2_policy": "inputs larger than L2",
+                   "parallelism": f"dp{world} (by prompt group, no data-path collective)"},
+        "clocks": clocks, "e2e": None, "gpu_launches": 4 * args.steps,
+        "roofline": {"bound": "hbm", "kernel": "onpolicy_rows_kernel", "achieved": ach, "peak": peak,
+                     "peak_kind": peak_kind, "unit": "GB/s", "frac": ach / peak, "frac_of_8TBs_nominal": ach / 8000.0,
+                     "algorithmic_bytes_per_launch": algo, "traffic": None},
+        "cpu_baseline": None, "stats": {"loss": st["loss"], "status": st["status"]},
+    }
+    print(json.dumps(line), flush=True)
+    if dist:
+        dist.destroy_process_group()
+
+
 # DRAM traffic of pass 2 per algorithmic byte, from the ncu capture summarised under profiles/
 # (dram__bytes_read.sum + dram__bytes_write.sum of a smaller launch, which scales with rows).
 TRAFFIC_P2_PER_BYTE = 0.9735
@@ -582,7 +681,7 @@ def main():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="slm", choices=["slm", "fused"],
+    ap.add_argument("--workload", default="slm", choices=["slm", "fused", "onpolicy"],
                     help="slm: the logits-in path the metric is quoted on (default); fused: the LM-head form")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--skip-e2e", action="store_true", help="leave out the host-buffer leg (profiling)")
@@ -596,6 +695,8 @@ def main():
         args.warmup = max(args.warmup, 3)
         if args.workload == "fused":
             run_fused(args)
+        elif args.workload == "onpolicy":
+            run_onpolicy(args)
         else:
             run_ours(args)
 

@@ -243,6 +243,32 @@ rapid_status_t rapid_pg_dlogits_chunk(const rapid_desc_t* desc, const void* logi
                                       void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The on-policy special case in a single pass over the logits.  When the behaviour policy IS the
+ * current policy (mu = pi_theta: the first inner step after Algorithm 1 refreshes mu, and every
+ * step of the plain policy-gradient baseline) every importance weight is 1, Eq. 3 reduces to
+ * Eq. 1 and Eq. 5 to the group advantage of Eq. 2, which needs rewards only.  The coefficient
+ * g_n = A_n / Z is then known before any logit is read, so each row is read once from memory
+ * (its second sweep is served from L2) and written once:
+ *
+ *   A_n = R_n - (1/N_k) sum_{n' in group k} R_n'          Eq. 2 (leave-one-out by flag)
+ *   loss = - sum_n g_n sum_t m_r log pi_theta(y_t),       Eq. 1
+ *   dlogits[r, v] = g_n m_r (softmax(z[r, .])_v - 1[v == y_r])
+ *
+ * Arguments as for rapid_pg_loss_fwd_bwd, without behav_logp; desc->eta and
+ * RAPID_FLAG_OUTER_UNCLIPPED have no effect.  dlogits may be the logits buffer itself.  Rows that
+ * are masked are never read; rows of a generation with g_n = 0 (for instance a prompt whose
+ * generations all earned the same reward) are read only if token_logp is requested.
+ * stats: n_clipped = 0 and both staleness means are 0 by definition.  A bounded wait that gives
+ * up raises stats->status to RAPID_ERR_TIMEOUT.
+ */
+rapid_status_t rapid_pg_loss_onpolicy_fwd_bwd(const rapid_desc_t* desc, const void* logits,
+                                              const int32_t* targets, const uint8_t* mask,
+                                              const float* rewards, const int32_t* group_offsets,
+                                              void* dlogits, float* loss, float* token_logp,
+                                              float* adv, rapid_stats_t* stats, void* workspace,
+                                              size_t workspace_bytes, void* stream);
+
+/*
  * The fused LM-head form: the logits z = hidden * w_vocab are formed tile by tile on the tensor
  * cores and never written to memory (this form comes from the benchmark definition; in the paper
  * the logits are simply the policy network's output, Sec. 3.1).  Computes the same loss as

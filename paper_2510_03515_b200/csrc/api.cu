@@ -184,4 +184,29 @@ rapid_status_t rapid_pg_loss_fwd_bwd(const rapid_desc_t* desc, const void* logit
                                   workspace_bytes, stream);
 }
 
+rapid_status_t rapid_pg_loss_onpolicy_fwd_bwd(const rapid_desc_t* desc, const void* logits,
+                                              const int32_t* targets, const uint8_t* mask,
+                                              const float* rewards, const int32_t* group_offsets,
+                                              void* dlogits, float* loss, float* token_logp, float* adv,
+                                              rapid_stats_t* stats, void* workspace,
+                                              size_t workspace_bytes, void* stream) {
+    rapid_status_t s = check_desc_full(desc);
+    if (s != RAPID_OK) return s;
+    if (!logits || !targets || !rewards || !group_offsets || !dlogits || !loss) return RAPID_ERR_INVALID_ARG;
+    if (!aligned(logits, 16) || !aligned(dlogits, 16)) return RAPID_ERR_ALIGNMENT;
+    const int64_t T = (int64_t)desc->n_seq * desc->seq_len;
+    if (logits != dlogits) {
+        const size_t span = (size_t)T * (size_t)desc->ld * elem_size(desc->dtype);
+        const uintptr_t a = reinterpret_cast<uintptr_t>(logits);
+        const uintptr_t b = reinterpret_cast<uintptr_t>(dlogits);
+        if (a < b + span && b < a + span) return RAPID_ERR_INVALID_ARG;
+    }
+    Workspace ws;
+    if ((s = check_workspace(desc, workspace, workspace_bytes, &ws)) != RAPID_OK) return s;
+    int sms = 0;
+    if ((s = check_device(&sms)) != RAPID_OK) return s;
+    return cuda_status(launch_onpolicy(*desc, logits, dlogits, targets, mask, rewards, group_offsets, loss,
+                                       token_logp, adv, stats, ws, sms, static_cast<cudaStream_t>(stream)));
+}
+
 }  // extern "C"

@@ -32,7 +32,7 @@ seq_reduce_kernel(int seq_len, const float* __restrict__ behav_logp,
         double lp = 0.0;
         if (st == ROW_OK) {
             lp = ws.token_logp[r];
-            s += lp - (double)behav_logp[r];
+            if (behav_logp) s += lp - (double)behav_logp[r];  // no behaviour policy: on-policy, s_n = 0
             S += lp;
             cnt += 1;
         } else if (st == ROW_BAD_TOKEN) {

@@ -1,0 +1,679 @@
+// The on-policy special case in ONE pass over the logits: mu = pi_theta, so every importance
+// weight is 1 and the estimator is the policy gradient of Eq. 1 with the group advantage of Eq. 2
+// (group relative policy gradient, Sec. 3.3).  This is the first inner step of IW-GRPG after the
+// behaviour policy has been refreshed (Algorithm 1, "mu <- pi_theta"), and every step of the
+// plain PG baseline.
+//
+// The advantage A_n = R_n - mean_group(R) needs rewards only, so the coefficient g_n = A_n / Z is
+// known before any logit is read and a row can be finished as soon as its own log-sum-exp is:
+// one HBM read and one write per live row instead of two reads and one write.
+//
+//   onpolicy_prep_kernel    Eq. 2 advantages, coefficients, token count           (one CTA)
+//   onpolicy_rows_kernel    per live row: sweep 1 streams the row through a shared-memory ring
+//                           (bulk copies) and accumulates max / sum of exponentials; sweep 2 streams
+//                           the same row again -- it was read microseconds ago and is asked to stay
+//                           in L2 (evict-last hint) -- turns it into dlogits in place in shared memory
+//                           and sends it out with bulk stores.  Dead rows (masked, invalid token,
+//                           zero coefficient) are zero-filled from a shared-memory zero buffer.
+//   onpolicy_loss_kernel    S_n = sum_t log pi(y_t), loss = - sum_n g_n S_n, statistics (one CTA)
+//
+// Every wait on a barrier is bounded; a wait that gives up raises RAPID_ERR_TIMEOUT in the
+// statistics block and never traps.
+#include "rapid_common.cuh"
+#include "tma_pipe.cuh"
+
+namespace rapid {
+
+namespace {
+
+constexpr int kConsumers = 256;
+constexpr int kConsumerWarps = kConsumers / 32;
+constexpr int kThreads = kConsumers + 32;  // + one producer warp
+constexpr int kChunk = 16384;              // bytes per stage
+constexpr int kStages = 6;
+constexpr int kMaxPending = 3;             // bulk stores that may still be reading their stage
+constexpr int kVecPerChunk = kChunk / 16;
+constexpr int kVecPerThread = kVecPerChunk / kConsumers;
+constexpr int kZeroBuf = 8192;
+constexpr int kPrepThreads = 256;
+
+// L2 cache policies for bulk copies
+__device__ __forceinline__ uint64_t policy_evict_last() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ void bulk_load_hint(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar,
+                                               uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::
+            "r"(smem_u32(smem_dst)),
+        "l"(gsrc), "r"(bytes), "r"(smem_u32(bar)), "l"(policy)
+        : "memory");
+}
+__device__ __forceinline__ void bulk_store_hint(void* gdst, const void* smem_src, uint32_t bytes, uint64_t policy) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;" ::"l"(gdst),
+                 "r"(smem_u32(smem_src)), "r"(bytes), "l"(policy)
+                 : "memory");
+}
+
+__device__ __forceinline__ void consumer_barrier() {
+    asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory");
+}
+// the same barrier, returning the OR of `flag` over all consumers: a uniform decision to leave
+__device__ __forceinline__ bool consumer_barrier_or(bool flag) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, 1, %2, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(out)
+        : "r"((uint32_t)flag), "n"(kConsumers)
+        : "memory");
+    return out != 0;
+}
+
+__device__ __forceinline__ uint16_t to_bf16_bits(float x) { return (uint16_t)(pack_bf16x2(x, 0.f) & 0xffffu); }
+
+// ---- before the pass: Eq. 2 advantages and coefficients ------------------------------------------------
+
+__global__ void __launch_bounds__(kPrepThreads)
+onpolicy_prep_kernel(int n_seq, int seq_len, int vocab, int n_groups, double norm_z, uint32_t flags,
+                     const float* __restrict__ rewards, const int32_t* __restrict__ group_offsets,
+                     const int32_t* __restrict__ targets, const uint8_t* __restrict__ mask,
+                     float* __restrict__ adv_out, Workspace ws) {
+    __shared__ int sh_bad, sh_empty;
+    __shared__ long long sh_tok[kPrepThreads / 32];
+    const int tid = threadIdx.x;
+    if (tid == 0) {
+        sh_bad = 0;
+        sh_empty = 0;
+    }
+    __syncthreads();
+    for (int k = tid; k <= n_groups; k += kPrepThreads) {
+        const int o = group_offsets[k];
+        bool bad = (k == 0 && o != 0) || (k == n_groups && o != n_seq) || o < 0 || o > n_seq;
+        if (k < n_groups) {
+            const int o1 = group_offsets[k + 1];
+            if (o1 < o) bad = true;
+            if (o1 == o) atomicAdd(&sh_empty, 1);
+        }
+        if (bad) atomicAdd(&sh_bad, 1);
+    }
+    // tokens that count (only needed as the normaliser with RAPID_FLAG_NORM_TOKENS)
+    long long tok = 0;
+    if ((flags & RAPID_FLAG_NORM_TOKENS) && !(flags & RAPID_FLAG_NORM_GIVEN)) {
+        const int64_t T = (int64_t)n_seq * seq_len;
+        for (int64_t r = tid; r < T; r += kPrepThreads) {
+            const bool on = mask ? (mask[r] != 0) : true;
+            const int32_t y = targets[r];
+            tok += (on && y >= 0 && y < vocab) ? 1 : 0;
+        }
+    }
+    tok = warp_sum(tok);
+    if ((tid & 31) == 0) sh_tok[tid >> 5] = tok;
+    __syncthreads();
+    tok = 0;
+    for (int w = 0; w < kPrepThreads / 32; ++w) tok += sh_tok[w];
+
+    if (sh_bad != 0) {
+        const float nanf_ = __int_as_float(0x7fc00000);
+        for (int n = tid; n < n_seq; n += kPrepThreads) {
+            ws.coef[n] = 0.0;
+            ws.coef_log2[n] = -INFINITY;
+            ws.adv[n] = (double)nanf_;
+            if (adv_out) adv_out[n] = nanf_;
+        }
+        if (tid == 0) {
+            ws.stats->status = RAPID_ERR_INVALID_ARG;
+            ws.stats->n_empty_group = 0;
+        }
+        return;
+    }
+    const double Z = (flags & RAPID_FLAG_NORM_GIVEN)    ? norm_z
+                     : (flags & RAPID_FLAG_NORM_TOKENS) ? (double)tok
+                                                        : (double)n_seq;
+    const bool loo = (flags & RAPID_FLAG_LEAVE_ONE_OUT) != 0;
+    // one thread per group, members in index order: the plain definition of Eq. 2
+    for (int k = tid; k < n_groups; k += kPrepThreads) {
+        const int lo = group_offsets[k], hi = group_offsets[k + 1];
+        const int Nk = hi - lo;
+        if (Nk == 0) continue;
+        double sum = 0.0;
+        for (int n = lo; n < hi; ++n) sum = __dadd_rn(sum, (double)rewards[n]);
+        for (int n = lo; n < hi; ++n) {
+            const double R = (double)rewards[n];
+            double a;
+            if (loo) {
+                double others = 0.0;
+                for (int q = lo; q < hi; ++q)
+                    if (q != n) others = __dadd_rn(others, (double)rewards[q]);
+                if (flags & RAPID_FLAG_LOO_LITERAL_DIVISOR) a = __dsub_rn(R, __ddiv_rn(others, (double)Nk));
+                else if (Nk > 1) a = __dsub_rn(R, __ddiv_rn(others, (double)(Nk - 1)));
+                else a = R;
+            } else {
+                a = __dsub_rn(R, __ddiv_rn(sum, (double)Nk));
+            }
+            const double g = (Z > 0.0) ? a / Z : 0.0;
+            ws.adv[n] = a;
+            ws.coef[n] = g;
+            ws.coef_log2[n] = (g != 0.0) ? log2(fabs(g)) : -INFINITY;
+            ws.weight[n] = 1.0;
+            ws.clipped_w[n] = 1.0;
+            if (adv_out) adv_out[n] = (float)a;
+        }
+    }
+    if (tid == 0) {
+        ws.stats->status = RAPID_OK;
+        ws.stats->n_empty_group = sh_empty;
+    }
+}
+
+// ---- the pass ------------------------------------------------------------------------------------------
+
+struct RowConstBf16 {
+    float c;         // -lse log2(e) + log2|g|
+    float g;
+    uint32_t sign2;  // sign of g on both halves of a packed pair
+    int y;
+};
+struct RowConstF32 {
+    float M, a, g;  // row max, lse - M, coefficient
+    int y;
+};
+
+// running (max, sum of exponentials) of one thread
+struct Acc {
+    float m, s0, s1;
+};
+
+__device__ __forceinline__ void acc_vec(Acc& a, const uint4 (&q)[kVecPerThread], int nvalid, RowConstBf16*) {
+    // bf16: chunk maximum with packed max, then one fused multiply-add and one MUFU exponential per element
+    uint32_t mx = 0xff80ff80u;  // (-inf, -inf)
+#pragma unroll
+    for (int j = 0; j < kVecPerThread; ++j)
+        if (j < nvalid) mx = bf16x2_max(mx, bf16x2_max(bf16x2_max(q[j].x, q[j].y), bf16x2_max(q[j].z, q[j].w)));
+    const float bm = fmaxf(bf16_lo(mx), bf16_hi(mx));
+    if (bm > a.m) {
+        const float f = ex2_approx((a.m - bm) * kLog2e);
+        a.s0 *= f;
+        a.s1 *= f;
+        a.m = bm;
+    }
+    const float nm = -a.m * kLog2e;
+#pragma unroll
+    for (int j = 0; j < kVecPerThread; ++j) {
+        if (j < nvalid) {
+            const uint32_t w[4] = {q[j].x, q[j].y, q[j].z, q[j].w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                a.s0 += ex2_approx(fmaf(bf16_lo(w[k]), kLog2e, nm));
+                a.s1 += ex2_approx(fmaf(bf16_hi(w[k]), kLog2e, nm));
+            }
+        }
+    }
+}
+__device__ __forceinline__ void acc_vec(Acc& a, const uint4 (&q)[kVecPerThread], int nvalid, RowConstF32*) {
+    float bm = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < kVecPerThread; ++j)
+        if (j < nvalid)
+            bm = fmaxf(bm, fmaxf(fmaxf(__uint_as_float(q[j].x), __uint_as_float(q[j].y)),
+                                 fmaxf(__uint_as_float(q[j].z), __uint_as_float(q[j].w))));
+    if (bm > a.m) {
+        const float f = expf(a.m - bm);
+        a.s0 *= f;
+        a.s1 *= f;
+        a.m = bm;
+    }
+#pragma unroll
+    for (int j = 0; j < kVecPerThread; ++j) {
+        if (j < nvalid) {
+            a.s0 += expf(__uint_as_float(q[j].x) - a.m) + expf(__uint_as_float(q[j].y) - a.m);
+            a.s1 += expf(__uint_as_float(q[j].z) - a.m) + expf(__uint_as_float(q[j].w) - a.m);
+        }
+    }
+}
+__device__ __forceinline__ void acc_scalar(Acc& a, float z, bool base2) {
+    if (z > a.m) {
+        const float f = base2 ? ex2_approx((a.m - z) * kLog2e) : expf(a.m - z);
+        a.s0 *= f;
+        a.s1 *= f;
+        a.m = z;
+    }
+    a.s0 += base2 ? ex2_approx((z - a.m) * kLog2e) : expf(z - a.m);
+}
+
+__device__ __forceinline__ uint4 dz_vec(uint4 z, int e0, const RowConstBf16& rc) {
+    uint32_t w[4] = {z.x, z.y, z.z, z.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const float lo = ex2_approx(fmaf(bf16_lo(w[k]), kLog2e, rc.c));
+        const float hi = ex2_approx(fmaf(bf16_hi(w[k]), kLog2e, rc.c));
+        uint32_t out = pack_bf16x2(lo, hi) ^ rc.sign2;
+        if (e0 + 2 * k == (rc.y & ~1)) {  // the sampled token: g (p_y - 1), formed in float
+            const float ps = (rc.y & 1) ? hi : lo;
+            const uint32_t b = to_bf16_bits((rc.g < 0.f ? -ps : ps) - rc.g);
+            out = (rc.y & 1) ? ((out & 0x0000ffffu) | (b << 16)) : ((out & 0xffff0000u) | b);
+        }
+        w[k] = out;
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+__device__ __forceinline__ uint4 dz_vec(uint4 zb, int e0, const RowConstF32& rc) {
+    const float z[4] = {__uint_as_float(zb.x), __uint_as_float(zb.y), __uint_as_float(zb.z), __uint_as_float(zb.w)};
+    uint32_t o[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        float v = rc.g * expf((z[k] - rc.M) - rc.a);
+        if (e0 + k == rc.y) v -= rc.g;
+        o[k] = __float_as_uint(v);
+    }
+    return make_uint4(o[0], o[1], o[2], o[3]);
+}
+__device__ __forceinline__ void dz_scalar(const void* zsm, void* orow, int e_in_chunk, int e, const RowConstBf16& rc) {
+    const float z = __uint_as_float(((uint32_t) static_cast<const uint16_t*>(zsm)[e_in_chunk]) << 16);
+    const float ps = ex2_approx(fmaf(z, kLog2e, rc.c));
+    float val = (rc.g < 0.f) ? -ps : ps;
+    if (e == rc.y) val -= rc.g;
+    static_cast<uint16_t*>(orow)[e] = to_bf16_bits(val);
+}
+__device__ __forceinline__ void dz_scalar(const void* zsm, void* orow, int e_in_chunk, int e, const RowConstF32& rc) {
+    const float z = static_cast<const float*>(zsm)[e_in_chunk];
+    float val = rc.g * expf((z - rc.M) - rc.a);
+    if (e == rc.y) val -= rc.g;
+    static_cast<float*>(orow)[e] = val;
+}
+
+// Which sweeps a row gets.  Decided from the inputs alone, identically by every thread.
+enum : int { ROWS_NONE = 0, ROWS_STATS = 1, ROWS_BOTH = 2 };
+__device__ __forceinline__ int row_plan(int64_t r, int seq_len, int vocab, const int32_t* targets,
+                                        const uint8_t* mask, const Workspace& ws, bool want_logp, uint8_t* state) {
+    const bool on = mask ? (mask[r] != 0) : true;
+    const int32_t y = targets[r];
+    if (!on) {
+        *state = ROW_MASKED;
+        return ROWS_NONE;
+    }
+    if (y < 0 || y >= vocab) {
+        *state = ROW_BAD_TOKEN;
+        return ROWS_NONE;
+    }
+    *state = ROW_OK;
+    if (ws.coef[(int)(r / seq_len)] != 0.0) return ROWS_BOTH;
+    return want_logp ? ROWS_STATS : ROWS_NONE;
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads)
+onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, int64_t ld, int vocab, int seq_len,
+                     int64_t n_rows, const int32_t* __restrict__ targets, const uint8_t* __restrict__ mask,
+                     int want_logp, Workspace ws) {
+    constexpr int ESIZE = (DT == RAPID_BF16) ? 2 : 4;
+    constexpr int PER = 16 / ESIZE;
+    constexpr bool kBase2 = (DT == RAPID_BF16);
+    using RowConst = typename std::conditional<DT == RAPID_BF16, RowConstBf16, RowConstF32>::type;
+
+    extern __shared__ __align__(128) uint8_t dyn[];  // kStages x kChunk ring, then kZeroBuf zeros
+    uint8_t* ring = dyn;
+    uint8_t* zeros = dyn + (size_t)kStages * kChunk;
+    __shared__ __align__(8) uint64_t full_bar[kStages];
+    __shared__ __align__(8) uint64_t empty_bar[kStages];
+    __shared__ int abort_flag;
+    __shared__ float sh_m[kConsumerWarps];
+    __shared__ double sh_s[kConsumerWarps];
+    __shared__ double sh_lse;
+    __shared__ float sh_M;
+    __shared__ float sh_zy;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], 1);
+        }
+        abort_flag = 0;
+        mbar_init_fence();
+    }
+    for (int i = tid; i < kZeroBuf / 16; i += kThreads) reinterpret_cast<uint4*>(zeros)[i] = make_uint4(0, 0, 0, 0);
+    fence_proxy_async_smem();
+    __syncthreads();
+    volatile int* abortp = &abort_flag;
+
+    const int load_bytes = ((vocab * ESIZE + 15) / 16) * 16;  // stays inside the row: the pitch is a multiple of 16
+    const int n_chunks = (load_bytes + kChunk - 1) / kChunk;
+    const int nvec_row = vocab / PER;
+    const int whole = nvec_row * 16;  // bytes of a row in whole vectors of real columns
+
+    if (warp == kConsumerWarps) {
+        // ------------------------------- producer -------------------------------------------
+        if (lane == 0) {
+            const uint64_t keep = policy_evict_last(), stream = policy_evict_first();
+            uint32_t it = 0;
+            bool ok = true;
+            for (int64_t r = blockIdx.x; r < n_rows && ok; r += gridDim.x) {
+                uint8_t st;
+                const int plan = row_plan(r, seq_len, vocab, targets, mask, ws, want_logp != 0, &st);
+                if (plan == ROWS_NONE) continue;
+                const uint8_t* src = static_cast<const uint8_t*>(logits) + (size_t)r * ld * ESIZE;
+                for (int sweep = 0; sweep < plan && ok; ++sweep) {
+                    // first sweep of a row that will be read again: ask L2 to keep it
+                    const uint64_t pol = (sweep == 0 && plan == ROWS_BOTH) ? keep : stream;
+                    for (int c = 0; c < n_chunks; ++c, ++it) {
+                        const int s = it % kStages;
+                        const uint32_t use = it / kStages;
+                        if (use > 0 && !mbar_wait_bounded(&empty_bar[s], (use & 1u) ^ 1u, abortp)) {
+                            ok = false;
+                            break;
+                        }
+                        const int bytes = min(kChunk, load_bytes - c * kChunk);
+                        mbar_arrive_expect_tx(&full_bar[s], (uint32_t)bytes);
+                        bulk_load_hint(ring + (size_t)s * kChunk, src + (size_t)c * kChunk, (uint32_t)bytes,
+                                       &full_bar[s], pol);
+                    }
+                }
+            }
+            if (!ok || *abortp) {
+                const uint32_t first = it > (uint32_t)kStages ? it - kStages : 0u;
+                for (uint32_t j = first; j < it; ++j) {
+                    const unsigned long long t0 = global_timer_ns();
+                    while (!mbar_try_wait(&full_bar[j % kStages], (j / kStages) & 1u))
+                        if (global_timer_ns() - t0 > kWaitLimitNs) break;
+                }
+            }
+        }
+    } else {
+        // ------------------------------- consumers ------------------------------------------
+        const uint64_t stream = policy_evict_first();
+        uint32_t it = 0;
+        bool ok = true;
+        // stages whose outgoing store may still be reading them, newest first (-1: nothing to release);
+        // only thread 0 uses this
+        int pend[kMaxPending];
+#pragma unroll
+        for (int k = 0; k < kMaxPending; ++k) pend[k] = -2;  // -2: no group at all
+        auto release = [&](int s) {
+            if (s >= 0) mbar_arrive(&empty_bar[s]);
+        };
+        // a new bulk group was committed for stage s (or -1 for a zero fill): the group committed
+        // kMaxPending groups earlier has finished reading by the time the wait returns
+        auto pushed = [&](int s) {
+            bulk_wait_read<kMaxPending>();
+            release(pend[kMaxPending - 1]);
+#pragma unroll
+            for (int k = kMaxPending - 1; k > 0; --k) pend[k] = pend[k - 1];
+            pend[0] = s;
+        };
+        // give back the oldest outstanding stage, waiting only for that one store
+        auto drain_one = [&]() {
+            if (pend[2] != -2) {
+                bulk_wait_read<2>();
+                release(pend[2]);
+                pend[2] = -2;
+            } else if (pend[1] != -2) {
+                bulk_wait_read<1>();
+                release(pend[1]);
+                pend[1] = -2;
+            } else if (pend[0] != -2) {
+                bulk_wait_read<0>();
+                release(pend[0]);
+                pend[0] = -2;
+            }
+        };
+        static_assert(kMaxPending == 3, "drain_one is written for three pending stores");
+
+        for (int64_t r = blockIdx.x; r < n_rows && ok; r += gridDim.x) {
+            uint8_t state;
+            const int plan = row_plan(r, seq_len, vocab, targets, mask, ws, want_logp != 0, &state);
+            uint8_t* orow = static_cast<uint8_t*>(dlogits) + (size_t)r * ld * ESIZE;
+            // rows without gradient get zeros, straight from the zero buffer (after the row has been
+            // read, if it is read at all: dlogits may be the logits buffer itself)
+            auto zero_row = [&]() {
+                if (tid == 0) {
+                    for (int o = 0; o < whole; o += kZeroBuf)
+                        bulk_store_hint(orow + o, zeros, (uint32_t)min(kZeroBuf, whole - o), stream);
+                    bulk_commit();
+                    pushed(-1);
+                } else if (nvec_row * PER + (tid - 1) < vocab) {
+                    if (ESIZE == 2) reinterpret_cast<uint16_t*>(orow)[nvec_row * PER + tid - 1] = 0;
+                    else reinterpret_cast<float*>(orow)[nvec_row * PER + tid - 1] = 0.f;
+                }
+            };
+            if (plan == ROWS_NONE) {
+                zero_row();
+                if (tid == 0) {
+                    ws.row_state[r] = state;
+                    ws.lse[r] = 0.0;
+                    ws.token_logp[r] = 0.0;
+                    ws.row_max[r] = 0.f;
+                }
+                continue;
+            }
+            const int y = targets[r];
+            // ---- sweep 1: max and sum of exponentials ----
+            Acc acc{-INFINITY, 0.f, 0.f};
+            for (int c = 0; c < n_chunks; ++c, ++it) {
+                const int s = it % kStages;
+                const bool got = mbar_wait_bounded(&full_bar[s], (it / kStages) & 1u, abortp);
+                const uint4* sv = reinterpret_cast<const uint4*>(ring + (size_t)s * kChunk);
+                const int v0 = c * kVecPerChunk;
+                const int nv = min(kVecPerChunk, nvec_row - v0);
+                if (got) {
+                    uint4 q[kVecPerThread];
+                    int nvalid = 0;
+#pragma unroll
+                    for (int j = 0; j < kVecPerThread; ++j) {
+                        const int v = tid + j * kConsumers;
+                        if (v < nv) {
+                            q[j] = sv[v];
+                            nvalid = j + 1;
+                        }
+                    }
+                    if (nvalid > 0) acc_vec(acc, q, nvalid, (RowConst*)nullptr);
+                    if (c == n_chunks - 1) {  // ragged tail: fewer than one vector of real columns
+                        const int e = nvec_row * PER + tid;
+                        if (e < vocab) {
+                            const int ei = e - v0 * PER;
+                            const float z = (ESIZE == 2)
+                                                ? __uint_as_float(((uint32_t) reinterpret_cast<const uint16_t*>(sv)[ei]) << 16)
+                                                : reinterpret_cast<const float*>(sv)[ei];
+                            acc_scalar(acc, z, kBase2);
+                        }
+                    }
+                    const int yi = y - v0 * PER;  // the sampled token's logit
+                    if (tid == 0 && yi >= 0 && yi < kVecPerChunk * PER)
+                        sh_zy = (ESIZE == 2) ? __uint_as_float(((uint32_t) reinterpret_cast<const uint16_t*>(sv)[yi]) << 16)
+                                             : reinterpret_cast<const float*>(sv)[yi];
+                }
+                if (consumer_barrier_or(!got || *abortp != 0)) {  // everyone has read the stage, or all leave
+                    ok = false;
+                    break;
+                }
+                if (tid == 0) {
+                    mbar_arrive(&empty_bar[s]);
+                    if (c < kMaxPending) drain_one();  // stages still held by the previous row's stores
+                }
+            }
+            if (!ok) break;
+            // ---- the row's log-sum-exp, in double ----
+            {
+                float m = acc.m, s = acc.s0 + acc.s1;
+                const float wm = warp_max(m);
+                s *= (m == wm) ? 1.f : (kBase2 ? ex2_approx((m - wm) * kLog2e) : expf(m - wm));
+                s = warp_sum(s);
+                if (lane == 0) {
+                    sh_m[warp] = wm;
+                    sh_s[warp] = (double)s;
+                }
+                consumer_barrier();
+                if (tid == 0) {
+                    float mm = sh_m[0];
+                    for (int w = 1; w < kConsumerWarps; ++w) mm = fmaxf(mm, sh_m[w]);
+                    double tot = 0.0;
+                    for (int w = 0; w < kConsumerWarps; ++w)
+                        if (sh_s[w] > 0.0) tot += sh_s[w] * exp((double)sh_m[w] - (double)mm);
+                    const double lse = (double)mm + log(tot);
+                    sh_lse = lse;
+                    sh_M = mm;
+                    ws.row_state[r] = ROW_OK;
+                    ws.lse[r] = lse;
+                    ws.token_logp[r] = (double)sh_zy - lse;
+                    ws.row_max[r] = mm;
+                }
+                consumer_barrier();
+            }
+            if (plan != ROWS_BOTH) {
+                zero_row();
+                continue;
+            }
+            // ---- sweep 2: dlogits, in place in the stage, out by bulk store ----
+            const int n = (int)(r / seq_len);
+            const double g = ws.coef[n];
+            RowConst rc;
+            if constexpr (DT == RAPID_BF16) {
+                rc.c = (float)fma(-sh_lse, kLog2eD, ws.coef_log2[n]);
+                rc.g = (float)g;
+                rc.sign2 = (g < 0.0) ? 0x80008000u : 0u;
+                rc.y = y;
+            } else {
+                rc.M = sh_M;
+                rc.a = (float)(sh_lse - (double)sh_M);
+                rc.g = (float)g;
+                rc.y = y;
+            }
+            for (int c = 0; c < n_chunks; ++c, ++it) {
+                const int s = it % kStages;
+                const bool got = mbar_wait_bounded(&full_bar[s], (it / kStages) & 1u, abortp);
+                uint4* sv = reinterpret_cast<uint4*>(ring + (size_t)s * kChunk);
+                const int v0 = c * kVecPerChunk;
+                const int nv = min(kVecPerChunk, nvec_row - v0);
+                if (got) {
+                    if (c == n_chunks - 1) {
+                        const int e = nvec_row * PER + tid;
+                        if (e < vocab) dz_scalar(sv, orow, e - v0 * PER, e, rc);
+                    }
+                    uint4 z[kVecPerThread];
+#pragma unroll
+                    for (int j = 0; j < kVecPerThread; ++j) {
+                        const int v = tid + j * kConsumers;
+                        if (v < nv) z[j] = sv[v];
+                    }
+#pragma unroll
+                    for (int j = 0; j < kVecPerThread; ++j) {
+                        const int v = tid + j * kConsumers;
+                        if (v < nv) sv[v] = dz_vec(z[j], (v0 + v) * PER, rc);
+                    }
+                    fence_proxy_async_smem();
+                }
+                if (consumer_barrier_or(!got || *abortp != 0)) {
+                    ok = false;
+                    break;
+                }
+                if (tid == 0) {
+                    if (nv > 0) {
+                        bulk_store_hint(orow + (size_t)c * kChunk, sv, (uint32_t)nv * 16u, stream);
+                        bulk_commit();
+                        pushed(s);
+                    } else {
+                        mbar_arrive(&empty_bar[s]);  // nothing to send from this stage
+                    }
+                }
+            }
+        }
+        if (tid == 0) bulk_wait_all<0>();
+    }
+    __syncthreads();
+    if (tid == 0 && abort_flag) atomicMax(&ws.stats->status, (int)RAPID_ERR_TIMEOUT);
+}
+
+// ---- after the pass: the loss and the statistics ---------------------------------------------------------
+
+__global__ void __launch_bounds__(kPrepThreads)
+onpolicy_loss_kernel(int n_seq, float* __restrict__ loss_out, rapid_stats_t* __restrict__ stats_out, Workspace ws) {
+    __shared__ double sh_d[kPrepThreads / 32];
+    __shared__ long long sh_l[kPrepThreads / 32];
+    __shared__ int sh_i[kPrepThreads / 32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    double loss = 0.0;
+    long long tokens = 0;
+    int bad = 0;
+    for (int n = tid; n < n_seq; n += kPrepThreads) {
+        loss -= ws.coef[n] * ws.seq_logp[n];
+        tokens += ws.seq_tokens[n];
+        bad += ws.seq_bad[n];
+    }
+    loss = warp_sum(loss);
+    tokens = warp_sum(tokens);
+    bad = warp_sum(bad);
+    if (lane == 0) {
+        sh_d[warp] = loss;
+        sh_l[warp] = tokens;
+        sh_i[warp] = bad;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        double L = 0.0;
+        long long tk = 0;
+        int bd = 0;
+        for (int w = 0; w < kPrepThreads / 32; ++w) {
+            L += sh_d[w];
+            tk += sh_l[w];
+            bd += sh_i[w];
+        }
+        rapid_stats_t st;
+        st.status = ws.stats->status;
+        st.n_empty_group = ws.stats->n_empty_group;
+        if (st.status == RAPID_ERR_INVALID_ARG) L = (double)__int_as_float(0x7fc00000);
+        st.n_tokens = tk;
+        st.n_clipped = 0;       // every weight is exactly 1
+        st.n_bad_token = bd;
+        st.mean_log_cw = 0.0;
+        st.mean_abs_log_cw = 0.0;
+        st.loss = L;
+        *ws.stats = st;
+        if (stats_out) *stats_out = st;
+        if (loss_out) *loss_out = (float)L;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_onpolicy(const rapid_desc_t& d, const void* logits, void* dlogits, const int32_t* targets,
+                            const uint8_t* mask, const float* rewards, const int32_t* group_offsets, float* loss,
+                            float* token_logp, float* adv, rapid_stats_t* stats, const Workspace& ws, int sm_count,
+                            cudaStream_t stream) {
+    const int64_t T = (int64_t)d.n_seq * d.seq_len;
+    onpolicy_prep_kernel<<<1, kPrepThreads, 0, stream>>>(d.n_seq, d.seq_len, d.vocab, d.n_groups, d.norm_z, d.flags,
+                                                        rewards, group_offsets, targets, mask, adv, ws);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    constexpr size_t smem = (size_t)kStages * kChunk + kZeroBuf;
+    const int want_logp = token_logp != nullptr;
+    auto go = [&](auto kern) -> cudaError_t {
+        cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err != cudaSuccess) return err;
+        int per_sm = 0;
+        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kThreads, smem);
+        if (err != cudaSuccess) return err;
+        if (per_sm < 1) per_sm = 1;
+        int64_t grid = (int64_t)sm_count * per_sm;
+        if (grid > T) grid = T;
+        kern<<<(unsigned)grid, kThreads, smem, stream>>>(logits, dlogits, d.ld, d.vocab, d.seq_len, T, targets, mask,
+                                                         want_logp, ws);
+        return cudaGetLastError();
+    };
+    e = (d.dtype == RAPID_BF16) ? go(onpolicy_rows_kernel<RAPID_BF16>) : go(onpolicy_rows_kernel<RAPID_F32>);
+    if (e != cudaSuccess) return e;
+    e = launch_seq_reduce(d, nullptr, token_logp, ws, stream);
+    if (e != cudaSuccess) return e;
+    onpolicy_loss_kernel<<<1, kPrepThreads, 0, stream>>>(d.n_seq, loss, stats, ws);
+    return cudaGetLastError();
+}
+
+}  // namespace rapid

@@ -144,4 +144,9 @@ cudaError_t launch_dlogits(const rapid_desc_t& d, const void* logits_chunk, void
                            rapid_stats_t* stats_user, const Workspace& ws, int sm_count,
                            cudaStream_t stream);
 
+cudaError_t launch_onpolicy(const rapid_desc_t& d, const void* logits, void* dlogits, const int32_t* targets,
+                            const uint8_t* mask, const float* rewards, const int32_t* group_offsets, float* loss,
+                            float* token_logp, float* adv, rapid_stats_t* stats, const Workspace& ws, int sm_count,
+                            cudaStream_t stream);
+
 }  // namespace rapid
