@@ -115,8 +115,19 @@ __device__ __forceinline__ void dz_scalar(const void* zsm, void* orow, int e_in_
     static_cast<float*>(orow)[e] = val;
 }
 
-__device__ __forceinline__ void consumer_barrier() {
-    asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory");
+// barrier over the consumer warps, returning the OR of `flag` over all of them: the decision to
+// leave after a timeout is taken by everyone together, so nobody is left waiting at a later barrier
+__device__ __forceinline__ bool consumer_barrier_or(bool flag) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, 1, %2, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(out)
+        : "r"((uint32_t)flag), "n"(kConsumers)
+        : "memory");
+    return out != 0;
 }
 
 __device__ __forceinline__ bool row_is_live(const Workspace& ws, int64_t r, int seq_len) {
@@ -243,7 +254,7 @@ dlogits_kernel(const void* logits, void* dlogits /* may alias logits */, int64_t
             for (int c = 0; c < n_chunks; ++c, ++it) {
                 const int s = it % kStages;
                 // A wait that gives up raises the abort flag; the thread still goes to the barrier
-                // below, after which every consumer sees the flag and leaves together.
+                // below, which ORs every consumer's view, so all leave together.
                 const bool got = mbar_wait_bounded(&full_bar[s], (it / kStages) & 1u, abortp);
                 uint4* sv = reinterpret_cast<uint4*>(ring + (size_t)s * kChunk);
                 const int v0 = c * kVecPerChunk;                  // first vector of the chunk in the row
@@ -268,8 +279,7 @@ dlogits_kernel(const void* logits, void* dlogits /* may alias logits */, int64_t
                     }
                     fence_proxy_async_smem();  // generic writes above -> asynchronous read below
                 }
-                consumer_barrier();
-                if (*abortp) {
+                if (consumer_barrier_or(!got || *abortp != 0)) {
                     ok = false;
                     break;
                 }

@@ -26,26 +26,54 @@ namespace rapid {
 
 namespace {
 
-constexpr int kConsumers = 256;
+#ifndef RAPID_OP_CONSUMERS
+#define RAPID_OP_CONSUMERS 256
+#endif
+#ifndef RAPID_OP_CHUNK
+#define RAPID_OP_CHUNK 16384
+#endif
+#ifndef RAPID_OP_STAGES
+#define RAPID_OP_STAGES 6
+#endif
+#ifndef RAPID_OP_HINTS
+#define RAPID_OP_HINTS 3  // see policy_evict_last() below; 3 measured best by a small margin
+#endif
+#ifndef RAPID_OP_MINBLOCKS
+#define RAPID_OP_MINBLOCKS 2
+#endif
+constexpr int kConsumers = RAPID_OP_CONSUMERS;
 constexpr int kConsumerWarps = kConsumers / 32;
 constexpr int kThreads = kConsumers + 32;  // + one producer warp
-constexpr int kChunk = 16384;              // bytes per stage
-constexpr int kStages = 6;
+constexpr int kChunk = RAPID_OP_CHUNK;     // bytes per stage
+constexpr int kStages = RAPID_OP_STAGES;
 constexpr int kMaxPending = 3;             // bulk stores that may still be reading their stage
+static_assert(kStages >= kMaxPending + 2, "the ring must keep cycling while stores are in flight");
+static_assert((kChunk / 16) % kConsumers == 0, "a chunk is a whole number of 16-byte vectors per consumer");
 constexpr int kVecPerChunk = kChunk / 16;
 constexpr int kVecPerThread = kVecPerChunk / kConsumers;
+constexpr int kVecPerWarp = kVecPerThread * 32;  // a warp's contiguous slice of a chunk, in 16-byte vectors
 constexpr int kZeroBuf = 8192;
 constexpr int kPrepThreads = 256;
 
 // L2 cache policies for bulk copies
+// RAPID_OP_HINTS: 0 = no preference anywhere; 1 = first sweep evict-last, everything else evict-first;
+// 2 = first sweep evict-last, the rest no preference; 3 = first sweep no preference, the rest evict-first
 __device__ __forceinline__ uint64_t policy_evict_last() {
     uint64_t p;
+#if RAPID_OP_HINTS == 1 || RAPID_OP_HINTS == 2
     asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+#else
+    asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
+#endif
     return p;
 }
 __device__ __forceinline__ uint64_t policy_evict_first() {
     uint64_t p;
+#if RAPID_OP_HINTS == 1 || RAPID_OP_HINTS == 3
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+#else
+    asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
+#endif
     return p;
 }
 __device__ __forceinline__ void bulk_load_hint(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar,
@@ -311,7 +339,7 @@ __device__ __forceinline__ int row_plan(int64_t r, int seq_len, int vocab, const
 }
 
 template <int DT>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, RAPID_OP_MINBLOCKS)
 onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, int64_t ld, int vocab, int seq_len,
                      int64_t n_rows, const int32_t* __restrict__ targets, const uint8_t* __restrict__ mask,
                      int want_logp, Workspace ws) {
@@ -336,7 +364,7 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&full_bar[s], 1);
-            mbar_init(&empty_bar[s], 1);
+            mbar_init(&empty_bar[s], kConsumerWarps);  // every consumer warp gives the stage back
         }
         abort_flag = 0;
         mbar_init_fence();
@@ -394,7 +422,7 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
         uint32_t it = 0;
         bool ok = true;
         // stages whose outgoing store may still be reading them, newest first (-1: nothing to release);
-        // only thread 0 uses this
+        // lane 0 of every warp keeps its own (bulk groups belong to the thread that commits them)
         int pend[kMaxPending];
 #pragma unroll
         for (int k = 0; k < kMaxPending; ++k) pend[k] = -2;  // -2: no group at all
@@ -428,7 +456,9 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
         };
         static_assert(kMaxPending == 3, "drain_one is written for three pending stores");
 
-        for (int64_t r = blockIdx.x; r < n_rows && ok; r += gridDim.x) {
+        // After a timeout a warp stops working (ok = false) but keeps walking the rows, so that it
+        // still meets the others at the next live row's barrier, where all agree to leave.
+        for (int64_t r = blockIdx.x; r < n_rows; r += gridDim.x) {
             uint8_t state;
             const int plan = row_plan(r, seq_len, vocab, targets, mask, ws, want_logp != 0, &state);
             uint8_t* orow = static_cast<uint8_t*>(dlogits) + (size_t)r * ld * ESIZE;
@@ -446,7 +476,7 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
                 }
             };
             if (plan == ROWS_NONE) {
-                zero_row();
+                if (ok) zero_row();
                 if (tid == 0) {
                     ws.row_state[r] = state;
                     ws.lse[r] = 0.0;
@@ -456,62 +486,70 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
                 continue;
             }
             const int y = targets[r];
-            // ---- sweep 1: max and sum of exponentials ----
+            // ---- sweep 1: max and sum of exponentials.  Each warp owns a contiguous slice of every
+            // chunk and gives the stage back on its own (the stage's barrier counts the warps), so no
+            // CTA-wide barrier is needed per chunk ----
             Acc acc{-INFINITY, 0.f, 0.f};
-            for (int c = 0; c < n_chunks; ++c, ++it) {
-                const int s = it % kStages;
-                const bool got = mbar_wait_bounded(&full_bar[s], (it / kStages) & 1u, abortp);
-                const uint4* sv = reinterpret_cast<const uint4*>(ring + (size_t)s * kChunk);
-                const int v0 = c * kVecPerChunk;
-                const int nv = min(kVecPerChunk, nvec_row - v0);
-                if (got) {
+            if (ok) {
+                for (int c = 0; c < n_chunks; ++c, ++it) {
+                    const int s = it % kStages;
+                    const bool got = mbar_wait_bounded(&full_bar[s], (it / kStages) & 1u, abortp);
+                    if (__any_sync(0xffffffffu, !got)) {
+                        ok = false;
+                        break;
+                    }
+                    const uint4* sv = reinterpret_cast<const uint4*>(ring + (size_t)s * kChunk);
+                    const int v0 = c * kVecPerChunk;
+                    const int nv = min(kVecPerChunk, nvec_row - v0);
                     uint4 q[kVecPerThread];
                     int nvalid = 0;
 #pragma unroll
                     for (int j = 0; j < kVecPerThread; ++j) {
-                        const int v = tid + j * kConsumers;
+                        const int v = warp * kVecPerWarp + j * 32 + lane;
                         if (v < nv) {
                             q[j] = sv[v];
                             nvalid = j + 1;
                         }
                     }
-                    if (nvalid > 0) acc_vec(acc, q, nvalid, (RowConst*)nullptr);
+                    float ztail = 0.f;
+                    bool has_tail = false;
                     if (c == n_chunks - 1) {  // ragged tail: fewer than one vector of real columns
                         const int e = nvec_row * PER + tid;
                         if (e < vocab) {
                             const int ei = e - v0 * PER;
-                            const float z = (ESIZE == 2)
-                                                ? __uint_as_float(((uint32_t) reinterpret_cast<const uint16_t*>(sv)[ei]) << 16)
-                                                : reinterpret_cast<const float*>(sv)[ei];
-                            acc_scalar(acc, z, kBase2);
+                            ztail = (ESIZE == 2)
+                                        ? __uint_as_float(((uint32_t) reinterpret_cast<const uint16_t*>(sv)[ei]) << 16)
+                                        : reinterpret_cast<const float*>(sv)[ei];
+                            has_tail = true;
                         }
                     }
                     const int yi = y - v0 * PER;  // the sampled token's logit
                     if (tid == 0 && yi >= 0 && yi < kVecPerChunk * PER)
                         sh_zy = (ESIZE == 2) ? __uint_as_float(((uint32_t) reinterpret_cast<const uint16_t*>(sv)[yi]) << 16)
                                              : reinterpret_cast<const float*>(sv)[yi];
+                    __syncwarp();  // the whole warp has its data in registers: the stage can go
+                    if (lane == 0) {
+                        mbar_arrive(&empty_bar[s]);
+                        if (c < kMaxPending) drain_one();  // stages still held by this warp's stores of the previous row
+                    }
+                    if (nvalid > 0) acc_vec(acc, q, nvalid, (RowConst*)nullptr);
+                    if (has_tail) acc_scalar(acc, ztail, kBase2);
                 }
-                if (consumer_barrier_or(!got || *abortp != 0)) {  // everyone has read the stage, or all leave
+            }
+            // ---- the row's log-sum-exp, in double; also where all warps agree to leave after a timeout ----
+            {
+                float m = acc.m, sm = acc.s0 + acc.s1;
+                const float wm = warp_max(m);
+                sm *= (m == wm) ? 1.f : (kBase2 ? ex2_approx((m - wm) * kLog2e) : expf(m - wm));
+                sm = warp_sum(sm);
+                if (lane == 0) {
+                    sh_m[warp] = wm;
+                    sh_s[warp] = (double)sm;
+                }
+                if (consumer_barrier_or(!ok || *abortp != 0)) {
                     ok = false;
                     break;
                 }
-                if (tid == 0) {
-                    mbar_arrive(&empty_bar[s]);
-                    if (c < kMaxPending) drain_one();  // stages still held by the previous row's stores
-                }
-            }
-            if (!ok) break;
-            // ---- the row's log-sum-exp, in double ----
-            {
-                float m = acc.m, s = acc.s0 + acc.s1;
-                const float wm = warp_max(m);
-                s *= (m == wm) ? 1.f : (kBase2 ? ex2_approx((m - wm) * kLog2e) : expf(m - wm));
-                s = warp_sum(s);
-                if (lane == 0) {
-                    sh_m[warp] = wm;
-                    sh_s[warp] = (double)s;
-                }
-                consumer_barrier();
                 if (tid == 0) {
                     float mm = sh_m[0];
                     for (int w = 1; w < kConsumerWarps; ++w) mm = fmaxf(mm, sh_m[w]);
@@ -532,7 +570,8 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
                 zero_row();
                 continue;
             }
-            // ---- sweep 2: dlogits, in place in the stage, out by bulk store ----
+            // ---- sweep 2: dlogits, in place in the warp's slice of the stage, out by the warp's own
+            // bulk store ----
             const int n = (int)(r / seq_len);
             const double g = ws.coef[n];
             RowConst rc;
@@ -547,46 +586,50 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
                 rc.g = (float)g;
                 rc.y = y;
             }
-            for (int c = 0; c < n_chunks; ++c, ++it) {
+            for (int c = 0; c < n_chunks && ok; ++c, ++it) {
                 const int s = it % kStages;
                 const bool got = mbar_wait_bounded(&full_bar[s], (it / kStages) & 1u, abortp);
-                uint4* sv = reinterpret_cast<uint4*>(ring + (size_t)s * kChunk);
-                const int v0 = c * kVecPerChunk;
-                const int nv = min(kVecPerChunk, nvec_row - v0);
-                if (got) {
-                    if (c == n_chunks - 1) {
-                        const int e = nvec_row * PER + tid;
-                        if (e < vocab) dz_scalar(sv, orow, e - v0 * PER, e, rc);
-                    }
-                    uint4 z[kVecPerThread];
-#pragma unroll
-                    for (int j = 0; j < kVecPerThread; ++j) {
-                        const int v = tid + j * kConsumers;
-                        if (v < nv) z[j] = sv[v];
-                    }
-#pragma unroll
-                    for (int j = 0; j < kVecPerThread; ++j) {
-                        const int v = tid + j * kConsumers;
-                        if (v < nv) sv[v] = dz_vec(z[j], (v0 + v) * PER, rc);
-                    }
-                    fence_proxy_async_smem();
-                }
-                if (consumer_barrier_or(!got || *abortp != 0)) {
+                if (__any_sync(0xffffffffu, !got)) {
                     ok = false;
                     break;
                 }
-                if (tid == 0) {
-                    if (nv > 0) {
-                        bulk_store_hint(orow + (size_t)c * kChunk, sv, (uint32_t)nv * 16u, stream);
+                uint4* sv = reinterpret_cast<uint4*>(ring + (size_t)s * kChunk);
+                const int v0 = c * kVecPerChunk;
+                const int nv = min(kVecPerChunk, nvec_row - v0);
+                if (c == n_chunks - 1) {
+                    const int e = nvec_row * PER + tid;
+                    if (e < vocab) dz_scalar(sv, orow, e - v0 * PER, e, rc);
+                }
+                uint4 z[kVecPerThread];
+#pragma unroll
+                for (int j = 0; j < kVecPerThread; ++j) {
+                    const int v = warp * kVecPerWarp + j * 32 + lane;
+                    if (v < nv) z[j] = sv[v];
+                }
+#pragma unroll
+                for (int j = 0; j < kVecPerThread; ++j) {
+                    const int v = warp * kVecPerWarp + j * 32 + lane;
+                    if (v < nv) sv[v] = dz_vec(z[j], (v0 + v) * PER, rc);
+                }
+                fence_proxy_async_smem();  // generic writes above -> asynchronous read below
+                __syncwarp();
+                if (lane == 0) {
+                    const int nvw = min(kVecPerWarp, nv - warp * kVecPerWarp);  // whole vectors in this warp's slice
+                    if (nvw > 0) {
+                        const size_t off = (size_t)warp * kVecPerWarp * 16;
+                        bulk_store_hint(orow + (size_t)c * kChunk + off, reinterpret_cast<uint8_t*>(sv) + off,
+                                        (uint32_t)nvw * 16u, stream);
                         bulk_commit();
                         pushed(s);
                     } else {
-                        mbar_arrive(&empty_bar[s]);  // nothing to send from this stage
+                        mbar_arrive(&empty_bar[s]);  // nothing to send from this slice
                     }
                 }
             }
         }
-        if (tid == 0) bulk_wait_all<0>();
+        // a warp that gave up in the middle of a row still owes nothing to a barrier: the others see
+        // the abort flag in their next wait
+        if (lane == 0) bulk_wait_all<0>();
     }
     __syncthreads();
     if (tid == 0 && abort_flag) atomicMax(&ws.stats->status, (int)RAPID_ERR_TIMEOUT);
