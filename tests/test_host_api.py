@@ -119,3 +119,50 @@ def test_missing_library_raises(monkeypatch):
     monkeypatch.setattr(rb, "LIB_PATH", "/nonexistent/librapid_pg.so")
     with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
         rb.lib()
+
+
+def test_onpolicy_argument_validation():
+    L = rb.lib()
+    good = rb.make_desc(4, 8, 64, 2, torch.bfloat16)
+    big = 1 << 40
+
+    def call(desc, logits=FAKE, dlogits=FAKE + (1 << 30), targets=FAKE, rewards=FAKE, go=FAKE, loss=FAKE,
+             ws=FAKE, ws_bytes=big):
+        return L.rapid_pg_loss_onpolicy_fwd_bwd(C.byref(desc), logits, targets, None, rewards, go, dlogits, loss,
+                                                None, None, None, ws, ws_bytes, None)
+
+    assert call(good, logits=None) == rb.RAPID_ERR_INVALID_ARG
+    assert call(good, rewards=None) == rb.RAPID_ERR_INVALID_ARG
+    assert call(good, loss=None) == rb.RAPID_ERR_INVALID_ARG
+    assert call(good, logits=FAKE + 4) == rb.RAPID_ERR_ALIGNMENT
+    assert call(good, dlogits=FAKE + 64) == rb.RAPID_ERR_INVALID_ARG       # partial overlap
+    assert call(good, ws=None) == rb.RAPID_ERR_WORKSPACE
+    assert call(good, ws_bytes=64) == rb.RAPID_ERR_WORKSPACE
+    assert call(rb.make_desc(4, 8, 64, 2, torch.bfloat16, ld=60)) == rb.RAPID_ERR_INVALID_ARG
+    assert call(rb.make_desc(4, 8, 60, 2, torch.bfloat16, ld=60)) == rb.RAPID_ERR_ALIGNMENT
+
+
+def test_fused_head_argument_validation():
+    L = rb.lib()
+    good = rb.make_desc(4, 8, 64, 2, torch.bfloat16)
+    big = 1 << 40
+    WS = 0x100000   # 1024-byte aligned
+
+    def call(desc, D=64, hidden=FAKE, w=FAKE, dh=FAKE, dW=FAKE, loss=FAKE, ws=WS, ws_bytes=big):
+        return L.rapid_pg_loss_fused_head(C.byref(desc), D, hidden, w, FAKE, None, FAKE, FAKE, FAKE, loss, dh, dW,
+                                          None, None, None, ws, ws_bytes, None)
+
+    assert call(good, hidden=None) == rb.RAPID_ERR_INVALID_ARG
+    assert call(good, dW=None) == rb.RAPID_ERR_INVALID_ARG
+    assert call(good, D=0) == rb.RAPID_ERR_INVALID_ARG
+    assert call(good, D=60) == rb.RAPID_ERR_ALIGNMENT                      # hidden pitch not 16-byte
+    assert call(good, w=FAKE + 8) == rb.RAPID_ERR_ALIGNMENT
+    assert call(good, ws=WS + 256) == rb.RAPID_ERR_WORKSPACE               # needs 1024-byte alignment
+    assert call(good, ws_bytes=1000) == rb.RAPID_ERR_WORKSPACE
+    assert call(rb.make_desc(4, 8, 64, 2, torch.float32)) == rb.RAPID_ERR_INVALID_ARG      # bf16 only
+    assert call(rb.make_desc(4, 8, 60, 2, torch.bfloat16, ld=60)) == rb.RAPID_ERR_ALIGNMENT
+    n = rb.rapid_fused_head_workspace_bytes(rb.make_desc(64, 256, 151936, 8, torch.bfloat16), 1536)
+    T, V = 64 * 256, 151936
+    assert T * ((V + 63) // 64 * 64) * 2 <= n <= T * ((V + 63) // 64 * 64) * 2 + 2 * 594 * T * 4 + 64 * T
+    with pytest.raises(rb.RapidError):
+        rb.rapid_fused_head_workspace_bytes(rb.make_desc(64, 256, 151936, 8, torch.float32), 1536)
