@@ -266,3 +266,16 @@ def test_shards_with_given_normaliser_add_up_to_the_whole_batch(flags):
     scale = max(abs(full["loss"]), 1e-3 * float(np.abs(full["coef"] * full["seq_logp"]).sum()))
     assert abs(loss_sum - full["loss"]) / scale <= 2e-3
     assert tok_sum == full["n_tokens"]
+
+
+def test_single_path_baseline_is_one_group():
+    """The single-path baseline of Sec. 3.3 (A = R - batch-mean reward) is the one-group case of the
+    group advantage: all N generations in one group."""
+    w = synth.Workload("onegroup", 1, 6, 7, 520, "bf16", 2.0, 4.0, "uniform", len_lo=2, behav_sigma=0.0,
+                       reward_mode="per_prompt", seed=13)
+    b = synth.make_batch(w)
+    b["rewards"] = torch.tensor([1.0, 0.0, 0.0, 1.0, 1.0, 0.0])
+    o, g = run_both(b, w.n_seq, w.seq_len)
+    compare(o, g, _dt(w), w.seq_len)
+    # sigma = 0: weights are 1 up to float32 rounding of the stored behaviour log-probs
+    np.testing.assert_allclose(g["adv"], b["rewards"].numpy() - 0.5, atol=1e-5)
