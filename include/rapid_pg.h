@@ -289,10 +289,13 @@ rapid_status_t rapid_pg_loss_onpolicy_fwd_bwd(const rapid_desc_t* desc, const vo
  *               columns beyond that are untouched
  *   token_logp, adv, stats: optional outputs as for rapid_pg_loss_fwd_bwd
  *   workspace   rapid_fused_head_workspace_bytes(desc, hidden_dim) bytes, 1024-byte aligned.  It
- *               holds, besides the per-row state, one bf16 copy of dlogits ([T, vocab] rounded up
- *               to 64 columns) and two floats per row per 256 vocabulary columns.
+ *               holds, besides the per-row state, two floats per row per 256 vocabulary columns
+ *               and a bf16 copy of dlogits for at most 16384 rows at a time ([rows, vocab rounded
+ *               up to 64 columns]): the backward part runs over the mini-batch in chunks of that
+ *               many rows, dW accumulating from chunk to chunk.
  *
- * Four tensor-core kernels run (forward statistics, dlogits, dhidden, dW), each a persistent grid
+ * Tensor-core kernels run for the forward statistics and, per chunk of rows, for dlogits, dhidden
+ * and dW (four GEMM-sized contractions over the mini-batch in all), each a persistent grid
  * with bounded waits: a wait that gives up raises stats->status to RAPID_ERR_TIMEOUT and leaves the
  * outputs unspecified.  Returns RAPID_ERR_CUDA if the driver cannot encode the tensor maps.
  */

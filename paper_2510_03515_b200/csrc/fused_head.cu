@@ -23,12 +23,16 @@ namespace {
 
 using namespace umma;
 
+// The backward part runs over at most this many rows at a time, which bounds the dlogits scratch
+// (rows x vocabulary in bf16) whatever the size of the mini-batch; dW accumulates across chunks.
+constexpr int64_t kHeadChunkRows = 16384;
+
 // Scratch of the fused-head call, carved after the ordinary workspace.
 struct HeadScratch {
     float* part_m;   // [n_tiles][T] running maximum of a row within one 256-column tile
     float* part_s;   // [n_tiles][T] sum of exp(z - part_m)
     float* zy;       // [T] the sampled token's logit
-    uint16_t* dz;    // [T][ldz] bf16
+    uint16_t* dz;    // [min(T, kHeadChunkRows)][ldz] bf16
     int* status;     // raised to RAPID_ERR_TIMEOUT by a kernel whose bounded wait ran out
     int64_t ldz;
     int n_tiles;
@@ -49,7 +53,7 @@ inline size_t carve_head(const rapid_desc_t& d, void* base, size_t off0, HeadScr
     s.part_m = reinterpret_cast<float*>(take(nt * T * 4));
     s.part_s = reinterpret_cast<float*>(take(nt * T * 4));
     s.zy = reinterpret_cast<float*>(take(T * 4));
-    s.dz = reinterpret_cast<uint16_t*>(take(T * ldz * 2));
+    s.dz = reinterpret_cast<uint16_t*>(take((T < (size_t)kHeadChunkRows ? T : (size_t)kHeadChunkRows) * ldz * 2));
     s.status = reinterpret_cast<int*>(take(256));
     s.ldz = (int64_t)ldz;
     s.n_tiles = (int)nt;
@@ -183,11 +187,12 @@ struct WarpStore {
         }
         return stage + (n & 1u) * 4096u;
     }
-    __device__ void commit(const CUtensorMap* map, uint8_t* buf, int x, int y) {
+    __device__ void commit(const CUtensorMap* map, uint8_t* buf, int x, int y, bool add = false) {
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) {
-            tma_store_2d(map, buf, x, y);
+            if (add) tma_reduce_add_2d(map, buf, x, y);
+            else tma_store_2d(map, buf, x, y);
             bulk_commit();
         }
         ++n;
@@ -208,7 +213,8 @@ struct DzStore {
         const double* coef_log2;
         const uint8_t* row_state;
         const int32_t* targets;
-        int T, V, seq_len;
+        int T, V, seq_len;  // T: rows of this chunk
+        int row0;           // global index of the chunk's first row (per-row arrays are global)
     };
     const Params& p;
     const int quarter, lane;
@@ -216,12 +222,13 @@ struct DzStore {
     __device__ DzStore(const Params& p_, uint8_t* stage, int q, int l) : p(p_), quarter(q), lane(l), st(stage, l) {}
 
     __device__ void tile(int m0, int n0, uint32_t taddr) {
-        const int row = m0 + quarter * 32 + lane;
+        const int row_in_chunk = m0 + quarter * 32 + lane;
+        const int row = p.row0 + row_in_chunk;
         const int ncols = min(BN, p.V - n0);
         float c = -INFINITY, g = 0.f;  // dead row: 2^-inf = 0 everywhere, nothing subtracted
         uint32_t sign2 = 0;
         int ycol = -1;
-        if (row < p.T && p.row_state[row] == ROW_OK) {
+        if (row_in_chunk < p.T && p.row_state[row] == ROW_OK) {
             const int n = row / p.seq_len;
             const double gd = p.coef[n];
             if (gd != 0.0) {
@@ -311,6 +318,7 @@ struct StoreF32 {  // dW
     struct Params {
         CUtensorMap map;  // [M, N] float, box 32 x 32
         int N;
+        int accumulate;  // add to what is there (second and later row chunks) instead of overwriting
     };
     const Params& p;
     const int quarter, lane;
@@ -328,7 +336,7 @@ struct StoreF32 {  // dW
             for (int k = 0; k < 8; ++k)
                 *reinterpret_cast<uint4*>(buf + swz128(lane, k)) =
                     make_uint4(r[4 * k], r[4 * k + 1], r[4 * k + 2], r[4 * k + 3]);
-            st.commit(&p.map, buf, n0 + c * 32, m0 + quarter * 32);
+            st.commit(&p.map, buf, n0 + c * 32, m0 + quarter * 32, p.accumulate != 0);
         }
     }
     __device__ void finish() { st.finish(); }
@@ -406,52 +414,71 @@ extern "C" rapid_status_t rapid_pg_loss_fused_head(
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
     // tensor maps (host structs, passed to the kernels by value)
-    CUtensorMap h_k, w_mn, w_k, h_mn, dz_k, dz_mn;
-    DzStore::Params dzp;
-    StoreBf16::Params dhp;
-    StoreF32::Params dwp;
-    bool ok = make_map_bf16(&h_k, hidden, T, D, D, BK, BM)              // A of forward: rows x K
-              && make_map_bf16(&w_mn, w_vocab, D, V, ld, 64, BK)        // B of forward: K x N
-              && make_map_bf16(&w_k, w_vocab, D, V, ld, BK, BN)         // B of dh: N(=D) x K(=V)
-              && make_map_bf16(&h_mn, hidden, T, D, D, 64, BK)          // A of dW: K(=T) x M(=D)
-              && make_map_bf16(&dz_k, hs.dz, T, V, hs.ldz, BK, BM)      // A of dh: rows x K(=V)
-              && make_map_bf16(&dz_mn, hs.dz, T, V, hs.ldz, 64, BK)     // B of dW: K(=T) x N(=V)
-              && make_map_bf16(&dzp.map, hs.dz, T, V, hs.ldz, 64, 32)   // stores
-              && make_map_bf16(&dhp.map, dhidden, T, D, D, 64, 32) &&
-              make_map_f32(&dwp.map, dW, D, V, ld, 32, 32);
+    CUtensorMap h_k, w_mn, w_k;
+    bool ok = make_map_bf16(&h_k, hidden, T, D, D, BK, BM)        // A of forward: rows x K
+              && make_map_bf16(&w_mn, w_vocab, D, V, ld, 64, BK)  // B of forward and recompute: K x N
+              && make_map_bf16(&w_k, w_vocab, D, V, ld, BK, BN);  // B of dh: N(=D) x K(=V)
     if (!ok) return RAPID_ERR_CUDA;
 
-    const int mT = (int)((T + BM - 1) / BM), nV = (V + BN - 1) / BN;
+    const int nV = (V + BN - 1) / BN;
     clear_status_kernel<<<1, 1, 0, st>>>(hs.status);
 
     // forward
-    FwdStats::Params fp{hs.part_m, hs.part_s, hs.zy, targets, (int)T, V};
-    Shape fwd{mT, nV, (D + BK - 1) / BK, M_FASTEST};
-    if (launch_gemm<FwdStats, false, true>(h_k, w_mn, fwd, sms, hs.status, fp, st) != cudaSuccess) return RAPID_ERR_CUDA;
+    {
+        FwdStats::Params fp{hs.part_m, hs.part_s, hs.zy, targets, (int)T, V};
+        Shape fwd{(int)((T + BM - 1) / BM), nV, (D + BK - 1) / BK, M_FASTEST};
+        if (launch_gemm<FwdStats, false, true>(h_k, w_mn, fwd, sms, hs.status, fp, st) != cudaSuccess)
+            return RAPID_ERR_CUDA;
+    }
     head_merge_kernel<<<(unsigned)((T + kMergeRows - 1) / kMergeRows), kMergeRows * kMergeSlices, 0, st>>>(
         T, V, hs.n_tiles, hs.part_m, hs.part_s, hs.zy, targets, mask, ws);
     if (cudaGetLastError() != cudaSuccess) return RAPID_ERR_CUDA;
     if (launch_seq_reduce(*desc, behav_logp, token_logp, ws, st) != cudaSuccess) return RAPID_ERR_CUDA;
     if (launch_finalize(*desc, rewards, group_offsets, loss, adv, stats, ws, st) != cudaSuccess) return RAPID_ERR_CUDA;
 
-    // backward: dz, then dh and dW
-    dzp.lse = ws.lse;
-    dzp.coef = ws.coef;
-    dzp.coef_log2 = ws.coef_log2;
-    dzp.row_state = ws.row_state;
-    dzp.targets = targets;
-    dzp.T = (int)T;
-    dzp.V = V;
-    dzp.seq_len = desc->seq_len;
-    if (launch_gemm<DzStore, false, true>(h_k, w_mn, fwd, sms, hs.status, dzp, st) != cudaSuccess) return RAPID_ERR_CUDA;
+    // backward, a chunk of rows at a time: dz (recompute), then dh for those rows and the chunk's
+    // contribution to dW (the first chunk overwrites dW, later ones add to it, in stream order)
+    for (int64_t r0 = 0; r0 < T; r0 += kHeadChunkRows) {
+        const int64_t R = (T - r0 < kHeadChunkRows) ? T - r0 : kHeadChunkRows;
+        const uint16_t* h_c = static_cast<const uint16_t*>(hidden) + (size_t)r0 * D;
+        uint16_t* dh_c = static_cast<uint16_t*>(dhidden) + (size_t)r0 * D;
+        CUtensorMap hc_k, hc_mn, dz_k, dz_mn;
+        DzStore::Params dzp;
+        StoreBf16::Params dhp;
+        StoreF32::Params dwp;
+        ok = make_map_bf16(&hc_k, h_c, R, D, D, BK, BM)                // A of recompute: rows x K
+             && make_map_bf16(&hc_mn, h_c, R, D, D, 64, BK)            // A of dW: K(=rows) x M(=D)
+             && make_map_bf16(&dz_k, hs.dz, R, V, hs.ldz, BK, BM)      // A of dh: rows x K(=V)
+             && make_map_bf16(&dz_mn, hs.dz, R, V, hs.ldz, 64, BK)     // B of dW: K(=rows) x N(=V)
+             && make_map_bf16(&dzp.map, hs.dz, R, V, hs.ldz, 64, 32)   // stores
+             && make_map_bf16(&dhp.map, dh_c, R, D, D, 64, 32) && make_map_f32(&dwp.map, dW, D, V, ld, 32, 32);
+        if (!ok) return RAPID_ERR_CUDA;
+        const int mR = (int)((R + BM - 1) / BM);
 
-    dhp.N = D;
-    Shape sdh{mT, (D + BN - 1) / BN, (V + BK - 1) / BK, N_FASTEST};
-    if (launch_gemm<StoreBf16, false, false>(dz_k, w_k, sdh, sms, hs.status, dhp, st) != cudaSuccess) return RAPID_ERR_CUDA;
+        dzp.lse = ws.lse;
+        dzp.coef = ws.coef;
+        dzp.coef_log2 = ws.coef_log2;
+        dzp.row_state = ws.row_state;
+        dzp.targets = targets;
+        dzp.T = (int)R;
+        dzp.V = V;
+        dzp.seq_len = desc->seq_len;
+        dzp.row0 = (int)r0;
+        Shape sdz{mR, nV, (D + BK - 1) / BK, M_FASTEST};
+        if (launch_gemm<DzStore, false, true>(hc_k, w_mn, sdz, sms, hs.status, dzp, st) != cudaSuccess)
+            return RAPID_ERR_CUDA;
 
-    dwp.N = V;
-    Shape sdw{(D + BM - 1) / BM, nV, (int)((T + BK - 1) / BK), M_FASTEST};
-    if (launch_gemm<StoreF32, true, true>(h_mn, dz_mn, sdw, sms, hs.status, dwp, st) != cudaSuccess) return RAPID_ERR_CUDA;
+        dhp.N = D;
+        Shape sdh{mR, (D + BN - 1) / BN, (V + BK - 1) / BK, N_FASTEST};
+        if (launch_gemm<StoreBf16, false, false>(dz_k, w_k, sdh, sms, hs.status, dhp, st) != cudaSuccess)
+            return RAPID_ERR_CUDA;
+
+        dwp.N = V;
+        dwp.accumulate = (r0 > 0) ? 1 : 0;
+        Shape sdw{(D + BM - 1) / BM, nV, (int)((R + BK - 1) / BK), M_FASTEST};
+        if (launch_gemm<StoreF32, true, true>(hc_mn, dz_mn, sdw, sms, hs.status, dwp, st) != cudaSuccess)
+            return RAPID_ERR_CUDA;
+    }
 
     publish_status_kernel<<<1, 1, 0, st>>>(hs.status, stats, ws.stats);
     return cudaGetLastError() == cudaSuccess ? RAPID_OK : RAPID_ERR_CUDA;

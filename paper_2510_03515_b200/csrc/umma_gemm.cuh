@@ -112,6 +112,13 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void*
                  : "memory");
 }
 
+// the same, adding the box to what global memory holds (element type taken from the tensor map)
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, const void* smem_src, int x, int y) {
+    asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];" ::"l"(map),
+                 "r"(smem_u32(smem_src)), "r"(x), "r"(y)
+                 : "memory");
+}
+
 // Byte offset, inside a 128-byte-swizzled box whose rows are 128 bytes, of 16-byte chunk `chunk`
 // (0..7) of row `row`: the chunk index is XORed with the row index modulo 8.
 __device__ __forceinline__ uint32_t swz128(int row, int chunk) {

@@ -218,3 +218,19 @@ def test_fused_head_full_size_config():
     assert abs(a - c) <= 1e-3 * max(abs(a), abs(c)) + 1e-2, (a, c)
     dead = (adv == 0).repeat_interleave(L)
     assert (dh[dead] == 0).all()
+
+
+def test_fused_head_more_rows_than_one_backward_chunk():
+    """18000 rows: the backward part runs as a chunk of 16384 rows and a ragged second one, whose
+    contribution is ADDED to dW; everything against the dense float64 oracle."""
+    w = synth.CONFIGS["fused"].scaled(n_prompts=3, group_size=3, seq_len=2000, vocab=600, hidden=64,
+                                      length_mode="uniform", len_lo=1500, reward_mode="per_prompt", seed=71)
+    b = synth.make_head(w)
+    b["rewards"] = torch.randn(w.n_seq, generator=torch.Generator().manual_seed(8))
+    o = oracle_head(b, w)
+    g = run_head(b, w, o["behav"])
+    compare_head(o, g, w)
+    # the second chunk's rows really contribute: dW restricted to the first chunk differs from the total
+    first = 16384
+    part = (o["h"][:first].T @ o["dz"][:first])
+    assert np.abs(part - o["dW"]).max() > 100 * 2.0 ** -6 * np.sqrt((o["h"][first:] ** 2).T @ (o["dz"][first:] ** 2)).mean()
