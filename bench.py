@@ -149,8 +149,8 @@ def oracle_sample(w: synth.Workload, target_seconds: float = 10.0):
     import oracle
     cores = oracle.max_threads()
 
-    def run(seq_len: int):
-        ws = w.scaled(n_prompts=1, seq_len=seq_len, len_lo=max(1, w.len_lo * seq_len // w.seq_len))
+    def run(seq_len: int, n_prompts: int = 1):
+        ws = w.scaled(n_prompts=n_prompts, seq_len=seq_len, len_lo=max(1, w.len_lo * seq_len // w.seq_len))
         b = synth.make_batch(ws)
         bits = synth.bits_numpy(b["logits"])
         tg, mk = b["targets"].numpy(), b["mask"].numpy()
@@ -169,6 +169,12 @@ def oracle_sample(w: synth.Workload, target_seconds: float = 10.0):
     seq_len = int(min(w.seq_len, max(16, 16 * target_seconds / max(dt, 1e-3))))
     seq_len = max(16, min(seq_len, w.seq_len))
     dt, ntok, ws = run(seq_len)
+    if seq_len == w.seq_len and dt < 0.5 * target_seconds:
+        # whole generations already: take more prompt groups (at most 4; drawing their logits on the
+        # host is what takes the wall-clock time, not the oracle)
+        k = int(min(w.n_prompts, 4, max(1, target_seconds // max(dt, 1e-3))))
+        if k > 1:
+            dt, ntok, ws = run(seq_len, k)
     return {"value": ntok / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"{ws.n_seq} generations x {ws.seq_len} padded tokens ({ntok} unmasked), "
                       f"V={ws.vocab} {ws.dtype}, float64 steps 1-6, {dt:.2f} s",
