@@ -234,3 +234,22 @@ def test_fused_head_more_rows_than_one_backward_chunk():
     first = 16384
     part = (o["h"][:first].T @ o["dz"][:first])
     assert np.abs(part - o["dW"]).max() > 100 * 2.0 ** -6 * np.sqrt((o["h"][first:] ** 2).T @ (o["dz"][first:] ** 2)).mean()
+
+
+def test_fused_head_bad_tokens_and_empty_generation():
+    """Token ids outside [0, V) count as masked and are reported; a generation with no unmasked
+    token has weight 1 and no gradient; an empty group is skipped."""
+    w = synth.CONFIGS["fused"].scaled(n_prompts=2, group_size=3, seq_len=10, vocab=304, hidden=64, seed=5)
+    b = synth.make_head(w)
+    b["targets"][3] = 304
+    b["targets"][17] = -5
+    b["mask"][20:30] = 0                                  # generation 2: nothing counts
+    b["rewards"] = torch.tensor([1.0, 0.0, 0.5, 0.0, 1.0, 1.0])
+    b["group_offsets"] = torch.tensor([0, 3, 3, 6], dtype=torch.int32)   # an empty group in the middle
+    w = w.scaled(n_prompts=3, group_size=2)               # three groups now; the same six generations
+    o = oracle_head(b, w)
+    g = run_head(b, w, o["behav"])
+    compare_head(o, g, w)
+    assert g["stats"]["n_bad_token"] == 2 and g["stats"]["n_empty_group"] == 1
+    assert g["stats"]["n_tokens"] == 60 - 10 - 2
+    assert np.all(g["dh"][20:30] == 0.0) and np.all(g["dh"][[3, 17]] == 0.0)
