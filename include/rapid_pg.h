@@ -221,11 +221,11 @@ rapid_status_t rapid_pg_loss_fwd_bwd_noalloc(const rapid_desc_t* desc, const voi
  * one from rapid_workspace_bytes(desc), shared by all three steps.  dlogits_chunk may alias
  * logits_chunk.
  *
- * The kernels move data with asynchronous bulk copies and wait for them on barriers; every such
- * wait is bounded (a few seconds).  A wait that gives up never traps: in the statistics pass the
- * row is marked and rapid_pg_finalize reports RAPID_ERR_TIMEOUT in stats->status with a NaN loss;
- * in the dlogits pass the status word of `stats` (optional; pass the struct that finalize wrote)
- * is raised to RAPID_ERR_TIMEOUT and the affected rows of dlogits are unspecified.
+ * The statistics pass uses ordinary vector loads and has no device-side wait.  The dlogits pass
+ * moves data with asynchronous bulk copies and waits for them on barriers; every such wait is
+ * bounded (a few seconds).  A wait that gives up never traps: the status word of `stats`
+ * (optional; pass the struct that finalize wrote) is raised to RAPID_ERR_TIMEOUT and the affected
+ * rows of dlogits are unspecified.
  */
 rapid_status_t rapid_pg_stats_chunk(const rapid_desc_t* desc, const void* logits_chunk,
                                     int64_t row0, int64_t n_rows, const int32_t* targets,
