@@ -6,10 +6,8 @@
 //
 // bf16 logits: one sweep, online max/sum per thread in float (base-2 exponentials on the MUFU
 // pipe), combined across the CTA in double.
-// fp32 logits: the tolerance on the loss is tight (a generation sums thousands of token
-// log-probs), so the row maximum is found first and the exponentials are then summed against
-// that exact maximum, four at a time in float and accumulated in double.  The second sweep of a
-// row hits L2.
+// fp32 logits: also one sweep, with the accurate exponential; the tolerance on the loss is tight (a
+// generation sums thousands of token log-probs), so threads are combined in double.
 #include "rapid_common.cuh"
 
 namespace rapid {
@@ -83,52 +81,51 @@ __device__ __forceinline__ void row_sweep_bf16(const uint16_t* row, int vocab, f
 
 // ---- fp32 ------------------------------------------------------------------------------------
 
-__device__ __forceinline__ float row_max_f32(const float* row, int vocab) {
+// One sweep, online: every thread keeps its own running maximum and the sum of accurate
+// exponentials against it, four at a time in float and accumulated in double (rescaled in double on
+// the rare occasions the maximum moves); threads are combined in double afterwards.  A generation's
+// weight sums thousands of token log-probs, so a bias of even 1e-8 per row would show.
+__device__ __forceinline__ void f32_batch(const float4* q, int n, float& m, double& s) {
+    float bm = -INFINITY;
+    for (int j = 0; j < n; ++j) bm = fmaxf(bm, fmaxf(fmaxf(q[j].x, q[j].y), fmaxf(q[j].z, q[j].w)));
+    if (bm > m) {
+        if (s > 0.0) s *= exp((double)m - (double)bm);
+        m = bm;
+    }
+    for (int j = 0; j < n; ++j)
+        s += (double)((expf(q[j].x - m) + expf(q[j].y - m)) + (expf(q[j].z - m) + expf(q[j].w - m)));
+}
+
+__device__ __forceinline__ void row_sweep_f32(const float* row, int vocab, float& m_out, double& s_out) {
     constexpr int U = 4;
     const int tid = threadIdx.x;
     const int nvec = vocab >> 2;
     const float4* rv = reinterpret_cast<const float4*>(row);
     float m = -INFINITY;
-    int v = tid;
-    for (; v + (U - 1) * kThreads < nvec; v += U * kThreads) {
-        float4 q[U];
-#pragma unroll
-        for (int j = 0; j < U; ++j) q[j] = __ldg(rv + v + j * kThreads);
-#pragma unroll
-        for (int j = 0; j < U; ++j) m = fmaxf(m, fmaxf(fmaxf(q[j].x, q[j].y), fmaxf(q[j].z, q[j].w)));
-    }
-    for (; v < nvec; v += kThreads) {
-        const float4 q = __ldg(rv + v);
-        m = fmaxf(m, fmaxf(fmaxf(q.x, q.y), fmaxf(q.z, q.w)));
-    }
-    const int e = (nvec << 2) + tid;
-    if (e < vocab) m = fmaxf(m, __ldg(row + e));
-    return m;
-}
-
-__device__ __forceinline__ double row_expsum_f32(const float* row, int vocab, float M) {
-    constexpr int U = 4;
-    const int tid = threadIdx.x;
-    const int nvec = vocab >> 2;
-    const float4* rv = reinterpret_cast<const float4*>(row);
-    double acc = 0.0;
+    double s = 0.0;
     int v = tid;
     for (; v + (U - 1) * kThreads < nvec; v += U * kThreads) {
         float4 q[U];
 #pragma unroll
         for (int j = 0; j < U; ++j) q[j] = __ldcs(rv + v + j * kThreads);
-#pragma unroll
-        for (int j = 0; j < U; ++j)
-            acc += (double)((expf(q[j].x - M) + expf(q[j].y - M)) +
-                            (expf(q[j].z - M) + expf(q[j].w - M)));
+        f32_batch(q, U, m, s);
     }
     for (; v < nvec; v += kThreads) {
-        const float4 q = __ldcs(rv + v);
-        acc += (double)((expf(q.x - M) + expf(q.y - M)) + (expf(q.z - M) + expf(q.w - M)));
+        float4 q[1];
+        q[0] = __ldcs(rv + v);
+        f32_batch(q, 1, m, s);
     }
-    const int e = (nvec << 2) + tid;
-    if (e < vocab) acc += (double)expf(__ldg(row + e) - M);
-    return acc;
+    const int e = (nvec << 2) + tid;  // ragged tail (vocab not a multiple of 4)
+    if (e < vocab) {
+        const float z = __ldg(row + e);
+        if (z > m) {
+            if (s > 0.0) s *= exp((double)m - (double)z);
+            m = z;
+        }
+        s += (double)expf(z - m);
+    }
+    m_out = m;
+    s_out = s;
 }
 
 // ---- kernel ----------------------------------------------------------------------------------
@@ -140,7 +137,6 @@ row_stats_kernel(const void* __restrict__ logits, int64_t ld, int vocab, int64_t
                  const uint8_t* __restrict__ mask, Workspace ws) {
     __shared__ float sh_m[kWarps];
     __shared__ double sh_s[kWarps];
-    __shared__ float sh_bcast;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
     for (int64_t i = blockIdx.x; i < n_rows; i += gridDim.x) {
@@ -185,22 +181,25 @@ row_stats_kernel(const void* __restrict__ logits, int64_t ld, int vocab, int64_t
             }
         } else {
             const float* row = static_cast<const float*>(logits) + i * ld;
-            float m = warp_max(row_max_f32(row, vocab));
-            if (lane == 0) sh_m[warp] = m;
+            float m;
+            double s;
+            row_sweep_f32(row, vocab, m, s);
+            const float wm = warp_max(m);
+            // a thread that saw nothing has m = -inf and s = 0
+            double sd = (s > 0.0) ? s * exp((double)m - (double)wm) : 0.0;
+            sd = warp_sum(sd);
+            if (lane == 0) {
+                sh_m[warp] = wm;
+                sh_s[warp] = sd;
+            }
             __syncthreads();
             if (tid == 0) {
                 float mm = sh_m[0];
                 for (int w = 1; w < kWarps; ++w) mm = fmaxf(mm, sh_m[w]);
-                sh_bcast = mm;
-            }
-            __syncthreads();
-            M = sh_bcast;
-            double s = warp_sum(row_expsum_f32(row, vocab, M));
-            if (lane == 0) sh_s[warp] = s;
-            __syncthreads();
-            if (tid == 0) {
                 double tot = 0.0;
-                for (int w = 0; w < kWarps; ++w) tot += sh_s[w];
+                for (int w = 0; w < kWarps; ++w)
+                    if (sh_s[w] > 0.0) tot += sh_s[w] * exp((double)sh_m[w] - (double)mm);
+                M = mm;
                 S = tot;
                 zy = (double)row[y];
             }
