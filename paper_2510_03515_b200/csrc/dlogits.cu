@@ -40,7 +40,11 @@ constexpr int kConsumerWarps = kConsumers / 32;
 constexpr int kThreads = kConsumers + 32;  // + one producer warp
 constexpr int kChunk = RAPID_P2_CHUNK;     // bytes per stage
 constexpr int kStages = RAPID_P2_STAGES;
-constexpr int kStoreDepth = kStages - 2;   // bulk stores allowed to be reading their stage
+#ifndef RAPID_P2_STOREDEPTH
+#define RAPID_P2_STOREDEPTH (RAPID_P2_STAGES / 2)  // measured best: three stages loading, three draining
+#endif
+constexpr int kStoreDepth = RAPID_P2_STOREDEPTH;  // bulk stores allowed to be reading their stage
+static_assert(kStoreDepth >= 1 && kStoreDepth <= kStages - 2, "leave at least two stages for loads");
 constexpr int kVecPerChunk = kChunk / 16;
 constexpr int kVecPerThread = kVecPerChunk / kConsumers;
 static_assert(kVecPerChunk % kConsumers == 0, "chunk must be a multiple of 16 B x consumers");
