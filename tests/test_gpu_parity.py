@@ -279,3 +279,43 @@ def test_single_path_baseline_is_one_group():
     compare(o, g, _dt(w), w.seq_len)
     # sigma = 0: weights are 1 up to float32 rounding of the stored behaviour log-probs
     np.testing.assert_allclose(g["adv"], b["rewards"].numpy() - 0.5, atol=1e-5)
+
+
+def test_runs_on_the_callers_stream():
+    """Work is enqueued on the stream handed over (here torch's current, non-default stream) and is
+    ordered after that stream's earlier work: the logits are produced on the same stream just before."""
+    w = synth.Workload("stream", 2, 3, 6, 2048, "bf16", 2.0, 3.0, "uniform", len_lo=2, behav_sigma=0.2,
+                       reward_mode="per_prompt", seed=37)
+    b = synth.make_batch(w)
+    dev = torch.device("cuda")
+    ref = rb.pg_loss(b["logits"].to(dev), b["targets"].to(dev), b["mask"].to(dev), torch.full((w.n_rows,), -7.0, device=dev),
+                     b["rewards"].to(dev), b["group_offsets"].to(dev), w.n_seq, w.seq_len)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    staged = b["logits"].to(dev)
+    tg, mk, rw, go = b["targets"].to(dev), b["mask"].to(dev), b["rewards"].to(dev), b["group_offsets"].to(dev)
+    bh = torch.full((w.n_rows,), -7.0, device=dev)
+    torch.cuda.synchronize()
+    with torch.cuda.stream(side):
+        z = torch.empty_like(staged)
+        for _ in range(20):                  # keep the stream busy, then produce the input on it
+            z.copy_(staged * 0.5)
+        z.copy_(staged)
+        got = rb.pg_loss(z, tg, mk, bh, rw, go, w.n_seq, w.seq_len)
+    side.synchronize()
+    assert got.loss.item() == ref.loss.item()
+    assert torch.equal(got.dlogits, ref.dlogits)
+
+
+def test_many_small_generations():
+    """5000 generations in 1250 groups: the per-generation and per-group steps loop well past one CTA."""
+    N, L, V = 5000, 2, 64
+    gen = torch.Generator().manual_seed(3)
+    b = {"logits": torch.randn((N * L, V), generator=gen),
+         "targets": torch.randint(0, V, (N * L,), generator=gen, dtype=torch.int64).to(torch.int32),
+         "mask": (torch.rand(N * L, generator=gen) < 0.8).to(torch.uint8),
+         "rewards": (torch.rand(N, generator=gen) < 0.5).float(),
+         "group_offsets": (torch.arange(1251) * 4).to(torch.int32),
+         "behav_noise": torch.randn(N * L, generator=gen) * 0.3}
+    o, g = run_both(b, N, L)
+    compare(o, g, torch.float32, L)
