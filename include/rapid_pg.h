@@ -279,7 +279,9 @@ rapid_status_t rapid_pg_loss_onpolicy_fwd_bwd(const rapid_desc_t* desc, const vo
  *   desc        dtype must be RAPID_BF16; desc->ld is the row pitch, in elements, of BOTH w_vocab
  *               and dW (>= vocab, a multiple of 8)
  *   hidden_dim  D, a multiple of 8
- *   hidden      [T, D] bf16, contiguous rows (pitch D), 16-byte aligned
+ *   hidden      [T, D] bf16, contiguous rows (pitch D), 16-byte aligned.  Every row must be finite,
+ *               masked ones too: they enter the products with a zero coefficient (unlike the
+ *               logits-in calls, which never read a masked row)
  *   w_vocab     [D, ld] bf16, 16-byte aligned
  *   targets, mask, behav_logp, rewards, group_offsets: as for rapid_pg_loss_fwd_bwd
  *   loss        [1] float out

@@ -228,6 +228,7 @@ struct DzStore {
         float c = -INFINITY, g = 0.f;  // dead row: 2^-inf = 0 everywhere, nothing subtracted
         uint32_t sign2 = 0;
         int ycol = -1;
+        bool live = false;       // the row has a gradient; otherwise exact zeros, whatever z holds
         if (row_in_chunk < p.T && p.row_state[row] == ROW_OK) {
             const int n = row / p.seq_len;
             const double gd = p.coef[n];
@@ -236,6 +237,7 @@ struct DzStore {
                 g = (float)gd;
                 sign2 = (gd < 0.0) ? 0x80008000u : 0u;
                 ycol = p.targets[row] - n0;
+                live = true;
             }
         }
 #pragma unroll 1
@@ -252,7 +254,7 @@ struct DzStore {
                 for (int j = 0; j < 16; ++j) {
                     const float lo = ex2_approx(fmaf(__uint_as_float(r[2 * j]), kLog2e, c));
                     const float hi = ex2_approx(fmaf(__uint_as_float(r[2 * j + 1]), kLog2e, c));
-                    o[j] = pack_bf16x2(lo, hi) ^ sign2;
+                    o[j] = (live ? pack_bf16x2(lo, hi) : 0u) ^ sign2;
                 }
                 if (ycol >= 0 && (ycol >> 5) == cc) {  // the sampled token: g (p_y - 1), formed in float
                     const int jj = ycol & 31;

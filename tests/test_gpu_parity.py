@@ -319,3 +319,34 @@ def test_many_small_generations():
          "behav_noise": torch.randn(N * L, generator=gen) * 0.3}
     o, g = run_both(b, N, L)
     compare(o, g, torch.float32, L)
+
+
+@pytest.mark.parametrize("form", ["two_pass", "on_policy"])
+def test_masked_rows_are_never_read(form):
+    """Masked rows may hold anything (here NaN): outputs are bit-identical to a clean run."""
+    w = synth.Workload("nanmask", 2, 3, 8, 4096, "bf16", 2.0, 3.0, "uniform", len_lo=2, behav_sigma=0.2,
+                       reward_mode="per_prompt", seed=43)
+    b = synth.make_batch(w)
+    dev = torch.device("cuda")
+    poisoned = b["logits"].clone()
+    poisoned[b["mask"] == 0] = float("nan")
+    bh = torch.full((w.n_rows,), -7.0, device=dev)
+    outs = []
+    for z in (b["logits"], poisoned):
+        if form == "two_pass":
+            r = rb.pg_loss(z.to(dev), b["targets"].to(dev), b["mask"].to(dev), bh, b["rewards"].to(dev),
+                           b["group_offsets"].to(dev), w.n_seq, w.seq_len)
+            outs.append((r.loss.item(), r.dlogits.clone()))
+        else:
+            desc = rb.make_desc(w.n_seq, w.seq_len, w.vocab, w.n_prompts, torch.bfloat16)
+            ws = rb.alloc_workspace(desc, dev)
+            loss = torch.zeros(1, device=dev)
+            dz = torch.empty((w.n_rows, w.vocab), dtype=torch.bfloat16, device=dev)
+            tl = torch.empty(w.n_rows, device=dev)
+            rb.rapid_pg_loss_onpolicy_fwd_bwd(desc, z.to(dev), b["targets"].to(dev), b["mask"].to(dev),
+                                              b["rewards"].to(dev), b["group_offsets"].to(dev), dz, loss, tl, None,
+                                              None, ws)
+            outs.append((loss.item(), dz.clone()))
+        torch.cuda.synchronize()
+    assert outs[0][0] == outs[1][0] and torch.equal(outs[0][1], outs[1][1])
+    assert torch.isfinite(outs[1][1].float()).all()

@@ -581,3 +581,83 @@ def test_head_functions_against_matmul_and_fd(oracle):
             Wm[d, v] -= eps
             fd_W[d, v] = (surrogate(h, Wp) - surrogate(h, Wm)) / (2 * eps)
     np.testing.assert_allclose(dW, fd_W, atol=1e-8)
+
+
+# --------------------------------------------------------------------------------------------
+# structural properties of the whole path (none of them is the oracle's own formula restated)
+# --------------------------------------------------------------------------------------------
+
+def _run(oracle, p, mu, logits=None, R=None, flags=0, eta=2.0, go=None, m=None):
+    return oracle.pg_loss(p["logits"] if logits is None else logits, p["N"], p["L"], p["V"], p["y"],
+                          p["m"] if m is None else m, mu, p["R"] if R is None else R,
+                          p["go"] if go is None else go, eta, flags, want_dlogits=True)
+
+
+def test_masked_rows_are_never_read(oracle):
+    """Whatever a masked row holds -- here NaN -- the result does not change, and its gradient is zero."""
+    p = _small_problem(seed=31)
+    mu = (-3.0 + 0.3 * p["rng"].normal(size=p["N"] * p["L"])).astype(np.float32)
+    a = _run(oracle, p, mu)
+    poisoned = p["logits"].copy()
+    poisoned[p["m"] == 0] = np.nan
+    b = _run(oracle, p, mu, logits=poisoned)
+    assert a["loss"] == b["loss"]
+    np.testing.assert_array_equal(a["dlogits"], b["dlogits"])
+    assert np.all(b["dlogits"][p["m"] == 0] == 0.0)
+
+
+def test_per_row_shift_of_the_logits_changes_nothing(oracle):
+    """softmax is invariant under adding a constant to a row: loss, weights and gradient stay put."""
+    p = _small_problem(seed=32)
+    mu = (-3.0 + 0.3 * p["rng"].normal(size=p["N"] * p["L"])).astype(np.float32)
+    a = _run(oracle, p, mu)
+    shift = (p["rng"].integers(-16, 16, (p["N"] * p["L"], 1)) / 4.0).astype(np.float32)  # exact in float32
+    b = _run(oracle, p, mu, logits=p["logits"] + shift)
+    assert b["loss"] == pytest.approx(a["loss"], rel=1e-12)
+    np.testing.assert_allclose(b["dlogits"], a["dlogits"], atol=1e-14)
+    np.testing.assert_allclose(b["weight"], a["weight"], rtol=1e-12)
+
+
+def test_permuting_generations_inside_a_group_permutes_the_result(oracle):
+    p = _small_problem(seed=33, N=6, sizes=(4, 2))
+    N, L, V = p["N"], p["L"], p["V"]
+    mu = (-3.0 + 0.3 * p["rng"].normal(size=N * L)).astype(np.float32)
+    a = _run(oracle, p, mu)
+    perm = np.array([2, 0, 3, 1, 5, 4])            # stays inside the groups {0..3} and {4, 5}
+    rows = (perm[:, None] * L + np.arange(L)[None, :]).reshape(-1)
+    q = dict(p, logits=p["logits"][rows], y=p["y"][rows], m=p["m"][rows], R=p["R"][perm])
+    b = _run(oracle, q, mu[rows])
+    assert b["loss"] == pytest.approx(a["loss"], rel=1e-12, abs=1e-15)
+    np.testing.assert_allclose(b["adv64"], a["adv64"][perm], atol=1e-15)
+    np.testing.assert_allclose(b["dlogits"], a["dlogits"][rows], atol=1e-15)
+
+
+def test_token_normaliser_only_rescales(oracle):
+    """Z = N versus Z = number of tokens: same direction, loss and gradient scaled by N / tokens."""
+    p = _small_problem(seed=34)
+    mu = (-3.0 + 0.3 * p["rng"].normal(size=p["N"] * p["L"])).astype(np.float32)
+    a = _run(oracle, p, mu, flags=0)
+    b = _run(oracle, p, mu, flags=2)
+    k = p["N"] / a["n_tokens"]
+    assert b["loss"] == pytest.approx(a["loss"] * k, rel=1e-12)
+    np.testing.assert_allclose(b["dlogits"], a["dlogits"] * k, rtol=1e-12, atol=1e-18)
+    np.testing.assert_array_equal(b["adv64"], a["adv64"])
+
+
+def test_rewards_shifted_by_a_constant_on_policy(oracle):
+    """Eq. 2 subtracts the group mean, so adding a constant to every reward of a group changes nothing
+    when all weights are one (it does off-policy, through the weighted baseline of Eq. 5)."""
+    p = _small_problem(seed=35, masked=False)
+    lp = oracle.token_logp(p["logits"], p["V"], p["y"], p["m"])["token_logp"]
+    A0 = oracle.group_advantage(p["R"], None, p["go"], 2.0)["adv64"]
+    A1 = oracle.group_advantage((p["R"] + np.float32(2.5)).astype(np.float32), None, p["go"], 2.0)["adv64"]
+    np.testing.assert_allclose(A1, A0, atol=1e-6)      # float32 rewards: the shift itself rounds
+    s = p["rng"].normal(0, 0.5, p["N"])
+    B0 = oracle.group_advantage(p["R"], s, p["go"], 2.0)["adv64"]
+    B1 = oracle.group_advantage((p["R"] + np.float32(2.5)).astype(np.float32), s, p["go"], 2.0)["adv64"]
+    c = np.minimum(np.exp(s), 2.0)
+    # off-policy the advantage moves by 2.5 (1 - mean_group(c))
+    go = p["go"]
+    expect = np.concatenate([np.full(go[k + 1] - go[k], 2.5 * (1.0 - c[go[k]:go[k + 1]].mean())) for k in range(len(go) - 1)])
+    np.testing.assert_allclose(B1 - B0, expect, atol=1e-6)
+    assert lp.shape[0] == p["N"] * p["L"]
