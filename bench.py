@@ -605,7 +605,7 @@ def run_onpolicy(args):
 
 # DRAM traffic of pass 2 per algorithmic byte, from the ncu capture summarised under profiles/
 # (dram__bytes_read.sum + dram__bytes_write.sum of a smaller launch, which scales with rows).
-TRAFFIC_P2_PER_BYTE = 0.9735
+TRAFFIC_P2_PER_BYTE = 0.9715
 
 
 def run_e2e(rb, args, desc, w, logits, tok, behav, dlogits, ws, loss, token_logp, adv, stats,
