@@ -350,3 +350,42 @@ def test_masked_rows_are_never_read(form):
         torch.cuda.synchronize()
     assert outs[0][0] == outs[1][0] and torch.equal(outs[0][1], outs[1][1])
     assert torch.isfinite(outs[1][1].float()).all()
+
+
+def test_two_pass_call_can_be_captured_in_a_cuda_graph():
+    """The library keeps no state and only enqueues kernels, so one rapid_pg_loss_fwd_bwd call can be
+    captured once and replayed (useful for small, launch-bound mini-batches): replays on fresh inputs
+    give the same bits as a direct call."""
+    w = synth.CONFIGS["tiny"]
+    b = synth.make_batch(w)
+    dev = torch.device("cuda")
+    z = b["logits"].to(dev)
+    tg, mk, rw, go = b["targets"].to(dev), b["mask"].to(dev), b["rewards"].to(dev), b["group_offsets"].to(dev)
+    bh = torch.full((w.n_rows,), -8.5, device=dev)
+    desc = rb.make_desc(w.n_seq, w.seq_len, w.vocab, w.n_prompts, torch.float32)
+    ws = rb.alloc_workspace(desc, dev)
+    out = {k: torch.zeros(s, device=dev) for k, s in (("loss", 1), ("tl", w.n_rows), ("adv", w.n_seq))}
+    dz = torch.zeros_like(z)
+    st = rb.alloc_stats(dev)
+
+    def call():
+        rb.rapid_pg_loss_fwd_bwd(desc, z, tg, mk, bh, rw, go, dz, out["loss"], out["tl"], out["adv"], st, ws)
+
+    call()                                   # warm-up outside capture (sets kernel attributes)
+    torch.cuda.synchronize()
+    direct = (out["loss"].item(), dz.clone())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        call()
+    for scale in (1.0, 0.5):
+        z.copy_(b["logits"].to(dev) * scale)
+        dz.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        if scale == 1.0:
+            assert out["loss"].item() == direct[0] and torch.equal(dz, direct[1])
+        else:
+            call_loss = out["loss"].item()
+            ref = rb.pg_loss(z, tg, mk, bh, rw, go, w.n_seq, w.seq_len)
+            torch.cuda.synchronize()
+            assert call_loss == ref.loss.item() and torch.equal(dz, ref.dlogits)
