@@ -14,25 +14,35 @@ namespace rapid {
 
 namespace {
 
-constexpr int kThreads = 256;
+#ifndef RAPID_P1_THREADS
+#define RAPID_P1_THREADS 128
+#endif
+#ifndef RAPID_P1_U
+#define RAPID_P1_U 8  // 16-byte loads in flight per thread (bf16 sweep)
+#endif
+constexpr int kThreads = RAPID_P1_THREADS;
 constexpr int kWarps = kThreads / 32;
 
 // ---- bf16 ------------------------------------------------------------------------------------
 
+// One batch of U vectors: the batch's exponentials are summed in float from zero and then added to
+// the thread's running sum in double.  (A float running sum silently drops terms below half an ulp
+// of the sum -- with a peaked softmax that is most of the tail -- and the lost mass shows up as a
+// bias of a few 1e-7 per token log-prob, which a generation-level weight then multiplies by its
+// length.)
 template <int U>
-__device__ __forceinline__ void bf16_batch(const uint4 (&q)[U], float& m, float& s0, float& s1) {
+__device__ __forceinline__ void bf16_batch(const uint4 (&q)[U], float& m, double& S) {
     uint32_t mx = bf16x2_max(bf16x2_max(q[0].x, q[0].y), bf16x2_max(q[0].z, q[0].w));
 #pragma unroll
     for (int j = 1; j < U; ++j)
         mx = bf16x2_max(mx, bf16x2_max(bf16x2_max(q[j].x, q[j].y), bf16x2_max(q[j].z, q[j].w)));
     const float bm = fmaxf(bf16_lo(mx), bf16_hi(mx));
     if (bm > m) {  // rare after the first few batches
-        const float f = ex2_approx((m - bm) * kLog2e);
-        s0 *= f;
-        s1 *= f;
+        S *= (double)ex2_approx((m - bm) * kLog2e);
         m = bm;
     }
     const float nm = -m * kLog2e;
+    float s0 = 0.f, s1 = 0.f;
 #pragma unroll
     for (int j = 0; j < U; ++j) {
         const uint32_t w[4] = {q[j].x, q[j].y, q[j].z, q[j].w};
@@ -42,41 +52,41 @@ __device__ __forceinline__ void bf16_batch(const uint4 (&q)[U], float& m, float&
             s1 += ex2_approx(fmaf(bf16_hi(w[k]), kLog2e, nm));
         }
     }
+    S += (double)(s0 + s1);
 }
 
 __device__ __forceinline__ void row_sweep_bf16(const uint16_t* row, int vocab, float& m_out,
-                                               float& s_out) {
-    constexpr int U = 4;
+                                               double& s_out) {
+    constexpr int U = RAPID_P1_U;
     const int tid = threadIdx.x;
     const int nvec = vocab >> 3;
     const uint4* rv = reinterpret_cast<const uint4*>(row);
-    float m = -INFINITY, s0 = 0.f, s1 = 0.f;
+    float m = -INFINITY;
+    double S = 0.0;
     int v = tid;
     for (; v + (U - 1) * kThreads < nvec; v += U * kThreads) {
         uint4 q[U];
 #pragma unroll
         for (int j = 0; j < U; ++j) q[j] = ld_stream(rv + v + j * kThreads);
-        bf16_batch<U>(q, m, s0, s1);
+        bf16_batch<U>(q, m, S);
     }
     for (; v < nvec; v += kThreads) {
         uint4 q[1];
         q[0] = ld_stream(rv + v);
-        bf16_batch<1>(q, m, s0, s1);
+        bf16_batch<1>(q, m, S);
     }
     // ragged tail (vocab not a multiple of 8): one element per thread
     const int e = (nvec << 3) + tid;
     if (e < vocab) {
         const float z = __uint_as_float(((uint32_t)row[e]) << 16);
         if (z > m) {
-            const float f = ex2_approx((m - z) * kLog2e);
-            s0 *= f;
-            s1 *= f;
+            S *= (double)ex2_approx((m - z) * kLog2e);
             m = z;
         }
-        s0 += ex2_approx((z - m) * kLog2e);
+        S += (double)ex2_approx((z - m) * kLog2e);
     }
     m_out = m;
-    s_out = s0 + s1;
+    s_out = S;
 }
 
 // ---- fp32 ------------------------------------------------------------------------------------
@@ -158,15 +168,16 @@ row_stats_kernel(const void* __restrict__ logits, int64_t ld, int vocab, int64_t
         double zy;
         if (DT == RAPID_BF16) {
             const uint16_t* row = static_cast<const uint16_t*>(logits) + i * ld;
-            float m, s;
+            float m;
+            double s;
             row_sweep_bf16(row, vocab, m, s);
             const float wm = warp_max(m);
             // a thread (or a whole warp, for a tiny vocabulary) that saw nothing has m = -inf, s = 0
-            s *= (m == wm) ? 1.f : ex2_approx((m - wm) * kLog2e);
+            if (m != wm) s *= (double)ex2_approx((m - wm) * kLog2e);
             s = warp_sum(s);
             if (lane == 0) {
                 sh_m[warp] = wm;
-                sh_s[warp] = (double)s;
+                sh_s[warp] = s;
             }
             __syncthreads();
             if (tid == 0) {
