@@ -26,19 +26,35 @@ constexpr int kWarps = kThreads / 32;
 // ---- bf16 ------------------------------------------------------------------------------------
 
 // One batch of U vectors: the batch's exponentials are summed in float from zero and then added to
-// the thread's running sum in double.  (A float running sum silently drops terms below half an ulp
-// of the sum -- with a peaked softmax that is most of the tail -- and the lost mass shows up as a
-// bias of a few 1e-7 per token log-prob, which a generation-level weight then multiplies by its
-// length.)
+// the thread's running sum with an error-compensated add (the rounding error of every add is kept in
+// a second float and folded back in at the end).  A plain float running sum silently drops terms
+// below half an ulp of the sum -- with a peaked softmax that is most of the tail -- and the lost mass
+// shows up as a bias of a few 1e-7 per token log-prob, which a generation-level weight then
+// multiplies by its length.  (A double running sum does the same job but costs 2-3 % on this part's
+// slow double-precision pipe.)
+struct FloatSum {
+    float s, c;  // running sum and the accumulated rounding error of its adds
+    __device__ __forceinline__ void add(float x) {  // requires s >= x >= 0 or s == 0: Fast2Sum
+        const float t = s + x;
+        c += (s - t) + x;
+        s = t;
+    }
+    __device__ __forceinline__ void scale(float f) {
+        s *= f;
+        c *= f;
+    }
+    __device__ __forceinline__ double value() const { return (double)s + (double)c; }
+};
+
 template <int U>
-__device__ __forceinline__ void bf16_batch(const uint4 (&q)[U], float& m, double& S) {
+__device__ __forceinline__ void bf16_batch(const uint4 (&q)[U], float& m, FloatSum& S) {
     uint32_t mx = bf16x2_max(bf16x2_max(q[0].x, q[0].y), bf16x2_max(q[0].z, q[0].w));
 #pragma unroll
     for (int j = 1; j < U; ++j)
         mx = bf16x2_max(mx, bf16x2_max(bf16x2_max(q[j].x, q[j].y), bf16x2_max(q[j].z, q[j].w)));
     const float bm = fmaxf(bf16_lo(mx), bf16_hi(mx));
     if (bm > m) {  // rare after the first few batches
-        S *= (double)ex2_approx((m - bm) * kLog2e);
+        S.scale(ex2_approx((m - bm) * kLog2e));
         m = bm;
     }
     const float nm = -m * kLog2e;
@@ -52,7 +68,14 @@ __device__ __forceinline__ void bf16_batch(const uint4 (&q)[U], float& m, double
             s1 += ex2_approx(fmaf(bf16_hi(w[k]), kLog2e, nm));
         }
     }
-    S += (double)(s0 + s1);
+    const float b = s0 + s1;
+    if (b > S.s) {  // keep the larger operand first, as Fast2Sum wants (early batches only)
+        const float old = S.s;
+        S.s = b;
+        S.add(old);
+    } else {
+        S.add(b);
+    }
 }
 
 __device__ __forceinline__ void row_sweep_bf16(const uint16_t* row, int vocab, float& m_out,
@@ -62,7 +85,7 @@ __device__ __forceinline__ void row_sweep_bf16(const uint16_t* row, int vocab, f
     const int nvec = vocab >> 3;
     const uint4* rv = reinterpret_cast<const uint4*>(row);
     float m = -INFINITY;
-    double S = 0.0;
+    FloatSum S{0.f, 0.f};
     int v = tid;
     for (; v + (U - 1) * kThreads < nvec; v += U * kThreads) {
         uint4 q[U];
@@ -76,17 +99,18 @@ __device__ __forceinline__ void row_sweep_bf16(const uint16_t* row, int vocab, f
         bf16_batch<1>(q, m, S);
     }
     // ragged tail (vocab not a multiple of 8): one element per thread
+    double tail = 0.0;
     const int e = (nvec << 3) + tid;
     if (e < vocab) {
         const float z = __uint_as_float(((uint32_t)row[e]) << 16);
         if (z > m) {
-            S *= (double)ex2_approx((m - z) * kLog2e);
+            S.scale(ex2_approx((m - z) * kLog2e));
             m = z;
         }
-        S += (double)ex2_approx((z - m) * kLog2e);
+        tail = (double)ex2_approx((z - m) * kLog2e);
     }
     m_out = m;
-    s_out = S;
+    s_out = S.value() + tail;
 }
 
 // ---- fp32 ------------------------------------------------------------------------------------
