@@ -253,3 +253,15 @@ def test_fused_head_bad_tokens_and_empty_generation():
     assert g["stats"]["n_bad_token"] == 2 and g["stats"]["n_empty_group"] == 1
     assert g["stats"]["n_tokens"] == 60 - 10 - 2
     assert np.all(g["dh"][20:30] == 0.0) and np.all(g["dh"][[3, 17]] == 0.0)
+
+
+@pytest.mark.parametrize("V,D,L", [(40, 8, 3), (8, 16, 1), (300 - 4, 24, 2)])
+def test_fused_head_shapes_smaller_than_one_tile(V, D, L):
+    """Vocabulary, hidden size and row count all below one 128 x 256 x 64 tile: the TMA boxes hang
+    over every edge of every matrix."""
+    w = synth.CONFIGS["fused"].scaled(n_prompts=1, group_size=3, seq_len=L, vocab=V, hidden=D, seed=90 + V)
+    b = synth.make_head(w)
+    b["rewards"] = torch.tensor([1.0, 0.0, -0.5])
+    o = oracle_head(b, w)
+    g = run_head(b, w, o["behav"])
+    compare_head(o, g, w)
