@@ -639,19 +639,27 @@ def run_e2e(rb, args, desc, w, logits, tok, behav, dlogits, ws, loss, token_logp
     h2d = nbytes + sum(v.numel() * v.element_size() for v in small.values()) + h_behav.numel() * 4
     d2h = 4
 
+    direct = host_logits.shape[0] == T   # the whole batch is pinned: let the kernels read it from there
+    if direct:
+        mode = "full pinned copy, read in place by the statistics pass (masked rows never cross the bus)"
+        h2d = n_tokens * logits.shape[1] * logits.element_size() + \
+            sum(v.numel() * v.element_size() for v in small.values()) + h_behav.numel() * 4
+
     def step():
-        if host_logits.shape[0] == T:
-            d_logits.copy_(host_logits, non_blocking=True)
+        for k in small:
+            d[k].copy_(small[k], non_blocking=True)
+        d_behav.copy_(h_behav, non_blocking=True)
+        if direct:
+            rb.rapid_pg_loss_fwd_bwd_hostlogits(desc, host_logits, d_logits, d["targets"], d["mask"], d_behav,
+                                                d["rewards"], d["group_offsets"], dlogits, loss, token_logp, adv,
+                                                stats, ws)
         else:
             R = host_logits.shape[0]
             for r0 in range(0, T, R):
                 n = min(R, T - r0)
                 d_logits[r0:r0 + n].copy_(host_logits[:n], non_blocking=True)
-        for k in small:
-            d[k].copy_(small[k], non_blocking=True)
-        d_behav.copy_(h_behav, non_blocking=True)
-        rb.rapid_pg_loss_fwd_bwd(desc, d_logits, d["targets"], d["mask"], d_behav, d["rewards"],
-                                 d["group_offsets"], dlogits, loss, token_logp, adv, stats, ws)
+            rb.rapid_pg_loss_fwd_bwd(desc, d_logits, d["targets"], d["mask"], d_behav, d["rewards"],
+                                     d["group_offsets"], dlogits, loss, token_logp, adv, stats, ws)
         h_loss.copy_(loss, non_blocking=True)
         torch.cuda.current_stream().synchronize()
         return float(h_loss[0])

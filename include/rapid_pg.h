@@ -243,6 +243,28 @@ rapid_status_t rapid_pg_dlogits_chunk(const rapid_desc_t* desc, const void* logi
                                       void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * rapid_pg_loss_fwd_bwd for logits that lie in page-locked HOST memory (cudaHostAlloc /
+ * cudaHostRegister, addressable by the device).  The statistics pass reads the rows straight from
+ * host memory over the bus -- masked rows are never transferred -- and leaves a copy of every row it
+ * read in `logits_staging`, which the dlogits pass then uses.  This is the one call whose `logits`
+ * argument is a host pointer; every other array is device memory as usual.
+ *   logits_host     [T, ld] host, page-locked; anything else (pageable host memory, a device
+ *                   pointer) returns RAPID_ERR_INVALID_ARG and enqueues nothing
+ *   logits_staging  [T, ld] device, same dtype and pitch; rows that are masked are left untouched
+ *   dlogits         [T, ld] device; may be logits_staging itself (in place)
+ * The other arguments, the results and the workspace are those of rapid_pg_loss_fwd_bwd.
+ * (Sec. 3.2 of the paper alternates inference and training on the same devices, so logits normally
+ * never leave the GPU; this form exists for pipelines that stage them through the host.)
+ */
+rapid_status_t rapid_pg_loss_fwd_bwd_hostlogits(const rapid_desc_t* desc, const void* logits_host,
+                                                void* logits_staging, const int32_t* targets,
+                                                const uint8_t* mask, const float* behav_logp,
+                                                const float* rewards, const int32_t* group_offsets,
+                                                void* dlogits, float* loss, float* token_logp,
+                                                float* adv, rapid_stats_t* stats, void* workspace,
+                                                size_t workspace_bytes, void* stream);
+
+/*
  * The on-policy special case in a single pass over the logits.  When the behaviour policy IS the
  * current policy (mu = pi_theta: the first inner step after Algorithm 1 refreshes mu, and every
  * step of the plain policy-gradient baseline) every importance weight is 1, Eq. 3 reduces to

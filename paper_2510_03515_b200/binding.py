@@ -40,7 +40,7 @@ EXPORTS = (
     "rapid_status_string", "rapid_version", "rapid_workspace_bytes", "rapid_group_advantage",
     "rapid_pg_loss_fwd_bwd", "rapid_pg_stats_chunk", "rapid_pg_finalize", "rapid_pg_dlogits_chunk",
     "rapid_pg_loss_fwd_bwd_noalloc", "rapid_fused_head_workspace_bytes", "rapid_pg_loss_fused_head",
-    "rapid_pg_loss_onpolicy_fwd_bwd",
+    "rapid_pg_loss_onpolicy_fwd_bwd", "rapid_pg_loss_fwd_bwd_hostlogits",
 )
 
 
@@ -90,6 +90,8 @@ def lib():
         L.rapid_pg_loss_fwd_bwd.argtypes = [dp] + [vp] * 12 + [sz, vp]
         L.rapid_pg_loss_fwd_bwd_noalloc.restype = C.c_int
         L.rapid_pg_loss_fwd_bwd_noalloc.argtypes = [dp] + [vp] * 12
+        L.rapid_pg_loss_fwd_bwd_hostlogits.restype = C.c_int
+        L.rapid_pg_loss_fwd_bwd_hostlogits.argtypes = [dp] + [vp] * 13 + [sz, vp]
         L.rapid_pg_loss_onpolicy_fwd_bwd.restype = C.c_int
         L.rapid_pg_loss_onpolicy_fwd_bwd.argtypes = [dp] + [vp] * 11 + [sz, vp]
         L.rapid_fused_head_workspace_bytes.restype = C.c_int
@@ -226,6 +228,19 @@ def rapid_pg_dlogits_chunk(desc: RapidDesc, logits_chunk: torch.Tensor,
     _check(lib().rapid_pg_dlogits_chunk(C.byref(desc), _ptr(logits_chunk), _ptr(dlogits_chunk),
                                         row0, n_rows, _ptr(targets), _ptr(stats), _ptr(workspace),
                                         workspace.numel(), _stream()), "rapid_pg_dlogits_chunk")
+
+
+def rapid_pg_loss_fwd_bwd_hostlogits(desc: RapidDesc, logits_host: torch.Tensor, logits_staging: torch.Tensor,
+                                     targets: torch.Tensor, mask: Optional[torch.Tensor],
+                                     behav_logp: torch.Tensor, rewards: torch.Tensor,
+                                     group_offsets: torch.Tensor, dlogits: torch.Tensor, loss: torch.Tensor,
+                                     token_logp: Optional[torch.Tensor], adv: Optional[torch.Tensor],
+                                     stats: Optional[torch.Tensor], workspace: torch.Tensor) -> None:
+    """`logits_host` is a PINNED CPU tensor; everything else lives on the device."""
+    _check(lib().rapid_pg_loss_fwd_bwd_hostlogits(
+        C.byref(desc), _ptr(logits_host), _ptr(logits_staging), _ptr(targets), _ptr(mask), _ptr(behav_logp),
+        _ptr(rewards), _ptr(group_offsets), _ptr(dlogits), _ptr(loss), _ptr(token_logp), _ptr(adv),
+        _ptr(stats), _ptr(workspace), workspace.numel(), _stream()), "rapid_pg_loss_fwd_bwd_hostlogits")
 
 
 def rapid_pg_loss_onpolicy_fwd_bwd(desc: RapidDesc, logits: torch.Tensor, targets: torch.Tensor,

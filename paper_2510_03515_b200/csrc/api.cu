@@ -184,6 +184,48 @@ rapid_status_t rapid_pg_loss_fwd_bwd(const rapid_desc_t* desc, const void* logit
                                   workspace_bytes, stream);
 }
 
+rapid_status_t rapid_pg_loss_fwd_bwd_hostlogits(const rapid_desc_t* desc, const void* logits_host,
+                                                void* logits_staging, const int32_t* targets,
+                                                const uint8_t* mask, const float* behav_logp,
+                                                const float* rewards, const int32_t* group_offsets,
+                                                void* dlogits, float* loss, float* token_logp, float* adv,
+                                                rapid_stats_t* stats, void* workspace,
+                                                size_t workspace_bytes, void* stream) {
+    rapid_status_t s = check_desc_full(desc);
+    if (s != RAPID_OK) return s;
+    if (!logits_host || !logits_staging || !targets || !behav_logp || !rewards || !group_offsets || !dlogits ||
+        !loss)
+        return RAPID_ERR_INVALID_ARG;
+    if (!aligned(logits_host, 16) || !aligned(logits_staging, 16) || !aligned(dlogits, 16)) return RAPID_ERR_ALIGNMENT;
+    const int64_t T = (int64_t)desc->n_seq * desc->seq_len;
+    if (logits_staging != dlogits) {
+        const size_t span = (size_t)T * (size_t)desc->ld * elem_size(desc->dtype);
+        const uintptr_t a = reinterpret_cast<uintptr_t>(logits_staging);
+        const uintptr_t b = reinterpret_cast<uintptr_t>(dlogits);
+        if (a < b + span && b < a + span) return RAPID_ERR_INVALID_ARG;
+    }
+    Workspace ws;
+    if ((s = check_workspace(desc, workspace, workspace_bytes, &ws)) != RAPID_OK) return s;
+    int sms = 0;
+    if ((s = check_device(&sms)) != RAPID_OK) return s;
+    // The kernel will dereference logits_host: it must be page-locked host memory that the device can
+    // address.  Anything else is refused here rather than left to fault on the device.
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, logits_host) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return RAPID_ERR_INVALID_ARG;
+    }
+    if (at.type != cudaMemoryTypeHost || !at.devicePointer) return RAPID_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = launch_row_stats(*desc, at.devicePointer, 0, T, targets, mask, ws, sms, st, logits_staging);
+    if (e != cudaSuccess) return RAPID_ERR_CUDA;
+    s = rapid_pg_finalize(desc, behav_logp, rewards, group_offsets, loss, token_logp, adv, stats, workspace,
+                          workspace_bytes, stream);
+    if (s != RAPID_OK) return s;
+    return rapid_pg_dlogits_chunk(desc, logits_staging, dlogits, 0, T, targets, stats, workspace,
+                                  workspace_bytes, stream);
+}
+
 rapid_status_t rapid_pg_loss_onpolicy_fwd_bwd(const rapid_desc_t* desc, const void* logits,
                                               const int32_t* targets, const uint8_t* mask,
                                               const float* rewards, const int32_t* group_offsets,

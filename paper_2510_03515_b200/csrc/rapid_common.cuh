@@ -129,7 +129,8 @@ __device__ __forceinline__ int warp_sum(int v) {
 // Host-side launchers (each enqueues on `stream` and returns the launch status).
 cudaError_t launch_row_stats(const rapid_desc_t& d, const void* logits_chunk, int64_t row0,
                              int64_t n_rows, const int32_t* targets, const uint8_t* mask,
-                             const Workspace& ws, int sm_count, cudaStream_t stream);
+                             const Workspace& ws, int sm_count, cudaStream_t stream,
+                             void* copy_out = nullptr);
 cudaError_t launch_seq_reduce(const rapid_desc_t& d, const float* behav_logp, float* token_logp_out,
                               const Workspace& ws, cudaStream_t stream);
 cudaError_t launch_finalize(const rapid_desc_t& d, const float* rewards,

@@ -78,12 +78,15 @@ __device__ __forceinline__ void bf16_batch(const uint4 (&q)[U], float& m, FloatS
     }
 }
 
+// `out`, when not null, receives a copy of the row (same layout): used when the logits are read from
+// host memory and the second pass wants them on the device.
 __device__ __forceinline__ void row_sweep_bf16(const uint16_t* row, int vocab, float& m_out,
-                                               double& s_out) {
+                                               double& s_out, uint16_t* out) {
     constexpr int U = RAPID_P1_U;
     const int tid = threadIdx.x;
     const int nvec = vocab >> 3;
     const uint4* rv = reinterpret_cast<const uint4*>(row);
+    uint4* ov = reinterpret_cast<uint4*>(out);
     float m = -INFINITY;
     FloatSum S{0.f, 0.f};
     int v = tid;
@@ -91,18 +94,25 @@ __device__ __forceinline__ void row_sweep_bf16(const uint16_t* row, int vocab, f
         uint4 q[U];
 #pragma unroll
         for (int j = 0; j < U; ++j) q[j] = ld_stream(rv + v + j * kThreads);
+        if (out) {
+#pragma unroll
+            for (int j = 0; j < U; ++j) ov[v + j * kThreads] = q[j];
+        }
         bf16_batch<U>(q, m, S);
     }
     for (; v < nvec; v += kThreads) {
         uint4 q[1];
         q[0] = ld_stream(rv + v);
+        if (out) ov[v] = q[0];
         bf16_batch<1>(q, m, S);
     }
     // ragged tail (vocab not a multiple of 8): one element per thread
     double tail = 0.0;
     const int e = (nvec << 3) + tid;
     if (e < vocab) {
-        const float z = __uint_as_float(((uint32_t)row[e]) << 16);
+        const uint16_t zb = row[e];
+        if (out) out[e] = zb;
+        const float z = __uint_as_float(((uint32_t)zb) << 16);
         if (z > m) {
             S.scale(ex2_approx((m - z) * kLog2e));
             m = z;
@@ -130,11 +140,13 @@ __device__ __forceinline__ void f32_batch(const float4* q, int n, float& m, doub
         s += (double)((expf(q[j].x - m) + expf(q[j].y - m)) + (expf(q[j].z - m) + expf(q[j].w - m)));
 }
 
-__device__ __forceinline__ void row_sweep_f32(const float* row, int vocab, float& m_out, double& s_out) {
+__device__ __forceinline__ void row_sweep_f32(const float* row, int vocab, float& m_out, double& s_out,
+                                              float* out) {
     constexpr int U = 4;
     const int tid = threadIdx.x;
     const int nvec = vocab >> 2;
     const float4* rv = reinterpret_cast<const float4*>(row);
+    float4* ov = reinterpret_cast<float4*>(out);
     float m = -INFINITY;
     double s = 0.0;
     int v = tid;
@@ -142,16 +154,22 @@ __device__ __forceinline__ void row_sweep_f32(const float* row, int vocab, float
         float4 q[U];
 #pragma unroll
         for (int j = 0; j < U; ++j) q[j] = __ldcs(rv + v + j * kThreads);
+        if (out) {
+#pragma unroll
+            for (int j = 0; j < U; ++j) ov[v + j * kThreads] = q[j];
+        }
         f32_batch(q, U, m, s);
     }
     for (; v < nvec; v += kThreads) {
         float4 q[1];
         q[0] = __ldcs(rv + v);
+        if (out) ov[v] = q[0];
         f32_batch(q, 1, m, s);
     }
     const int e = (nvec << 2) + tid;  // ragged tail (vocab not a multiple of 4)
     if (e < vocab) {
         const float z = __ldg(row + e);
+        if (out) out[e] = z;
         if (z > m) {
             if (s > 0.0) s *= exp((double)m - (double)z);
             m = z;
@@ -166,7 +184,7 @@ __device__ __forceinline__ void row_sweep_f32(const float* row, int vocab, float
 
 template <int DT>
 __global__ void __launch_bounds__(kThreads)
-row_stats_kernel(const void* __restrict__ logits, int64_t ld, int vocab, int64_t row0,
+row_stats_kernel(const void* __restrict__ logits, void* __restrict__ copy_out, int64_t ld, int vocab, int64_t row0,
                  int64_t n_rows, const int32_t* __restrict__ targets,
                  const uint8_t* __restrict__ mask, Workspace ws) {
     __shared__ float sh_m[kWarps];
@@ -194,7 +212,8 @@ row_stats_kernel(const void* __restrict__ logits, int64_t ld, int vocab, int64_t
             const uint16_t* row = static_cast<const uint16_t*>(logits) + i * ld;
             float m;
             double s;
-            row_sweep_bf16(row, vocab, m, s);
+            uint16_t* orow = copy_out ? static_cast<uint16_t*>(copy_out) + i * ld : nullptr;
+            row_sweep_bf16(row, vocab, m, s, orow);
             const float wm = warp_max(m);
             // a thread (or a whole warp, for a tiny vocabulary) that saw nothing has m = -inf, s = 0
             if (m != wm) s *= (double)ex2_approx((m - wm) * kLog2e);
@@ -212,13 +231,14 @@ row_stats_kernel(const void* __restrict__ logits, int64_t ld, int vocab, int64_t
                     tot += sh_s[w] * (double)ex2_approx((sh_m[w] - mm) * kLog2e);
                 M = mm;
                 S = tot;
-                zy = (double)__uint_as_float(((uint32_t)row[y]) << 16);
+                zy = (double)__uint_as_float(((uint32_t)row[y]) << 16);  // (one more 2-byte read of the row)
             }
         } else {
             const float* row = static_cast<const float*>(logits) + i * ld;
             float m;
             double s;
-            row_sweep_f32(row, vocab, m, s);
+            float* orow = copy_out ? static_cast<float*>(copy_out) + i * ld : nullptr;
+            row_sweep_f32(row, vocab, m, s, orow);
             const float wm = warp_max(m);
             // a thread that saw nothing has m = -inf and s = 0
             double sd = (s > 0.0) ? s * exp((double)m - (double)wm) : 0.0;
@@ -254,7 +274,7 @@ row_stats_kernel(const void* __restrict__ logits, int64_t ld, int vocab, int64_t
 
 cudaError_t launch_row_stats(const rapid_desc_t& d, const void* logits_chunk, int64_t row0,
                              int64_t n_rows, const int32_t* targets, const uint8_t* mask,
-                             const Workspace& ws, int sm_count, cudaStream_t stream) {
+                             const Workspace& ws, int sm_count, cudaStream_t stream, void* copy_out) {
     if (n_rows <= 0) return cudaSuccess;
     int per_sm = 0;
     cudaError_t e;
@@ -270,10 +290,10 @@ cudaError_t launch_row_stats(const rapid_desc_t& d, const void* logits_chunk, in
     if (grid > n_rows) grid = n_rows;
     if (d.dtype == RAPID_BF16)
         row_stats_kernel<RAPID_BF16><<<(unsigned)grid, kThreads, 0, stream>>>(
-            logits_chunk, d.ld, d.vocab, row0, n_rows, targets, mask, ws);
+            logits_chunk, copy_out, d.ld, d.vocab, row0, n_rows, targets, mask, ws);
     else
         row_stats_kernel<RAPID_F32><<<(unsigned)grid, kThreads, 0, stream>>>(
-            logits_chunk, d.ld, d.vocab, row0, n_rows, targets, mask, ws);
+            logits_chunk, copy_out, d.ld, d.vocab, row0, n_rows, targets, mask, ws);
     return cudaGetLastError();
 }
 

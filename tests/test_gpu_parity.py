@@ -389,3 +389,45 @@ def test_two_pass_call_can_be_captured_in_a_cuda_graph():
             ref = rb.pg_loss(z, tg, mk, bh, rw, go, w.n_seq, w.seq_len)
             torch.cuda.synchronize()
             assert call_loss == ref.loss.item() and torch.equal(dz, ref.dlogits)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_logits_read_from_pinned_host_memory(dtype):
+    """The host-logits form gives the same bits as copying the logits over first; rows that are
+    masked never reach the staging buffer; pointers that are not page-locked host memory are refused
+    before anything runs."""
+    import ctypes as C
+    w = synth.Workload("hostz", 2, 3, 9, 4100 if dtype == "f32" else 4104, dtype, 2.0, 3.0, "uniform", len_lo=3,
+                       behav_sigma=0.2, reward_mode="per_prompt", seed=47)
+    b = synth.make_batch(w)
+    dev = torch.device("cuda")
+    dt = synth.torch_dtype(w)
+    tg, mk, rw, go = b["targets"].to(dev), b["mask"].to(dev), b["rewards"].to(dev), b["group_offsets"].to(dev)
+    bh = torch.full((w.n_rows,), -7.5, device=dev)
+    ref = rb.pg_loss(b["logits"].to(dev), tg, mk, bh, rw, go, w.n_seq, w.seq_len)
+    torch.cuda.synchronize()
+
+    pinned = b["logits"].clone().pin_memory()
+    staging = torch.full_like(b["logits"], 7.0, device=dev)
+    desc = rb.make_desc(w.n_seq, w.seq_len, w.vocab, w.n_prompts, dt)
+    ws = rb.alloc_workspace(desc, dev)
+    loss = torch.zeros(1, device=dev)
+    dz = torch.empty_like(staging)
+    tl = torch.empty(w.n_rows, device=dev)
+    adv = torch.empty(w.n_seq, device=dev)
+    st = rb.alloc_stats(dev)
+    rb.rapid_pg_loss_fwd_bwd_hostlogits(desc, pinned, staging, tg, mk, bh, rw, go, dz, loss, tl, adv, st, ws)
+    torch.cuda.synchronize()
+    assert loss.item() == ref.loss.item() and torch.equal(dz, ref.dlogits) and torch.equal(tl, ref.token_logp)
+    on = b["mask"].bool()
+    assert torch.equal(staging[on.to(dev)].cpu(), b["logits"][on])          # what was read is what was staged
+    assert torch.all(staging[(~on).to(dev)] == 7.0)                          # masked rows never came over
+    assert rb.read_stats(st)["status"] == 0
+
+    L = rb.lib()
+    args = lambda z: (C.byref(desc), z, staging.data_ptr(), tg.data_ptr(), mk.data_ptr(), bh.data_ptr(), rw.data_ptr(),
+                      go.data_ptr(), dz.data_ptr(), loss.data_ptr(), None, None, None, ws.data_ptr(), ws.numel(), None)
+    pageable = b["logits"].clone()
+    assert L.rapid_pg_loss_fwd_bwd_hostlogits(*args(pageable.data_ptr())) == rb.RAPID_ERR_INVALID_ARG
+    assert L.rapid_pg_loss_fwd_bwd_hostlogits(*args(staging.data_ptr())) == rb.RAPID_ERR_INVALID_ARG
+    torch.cuda.synchronize()
