@@ -230,9 +230,12 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=dev)
     rb.lib()
 
-    w = synth.CONFIGS[WORKLOAD].scaled(seed=synth.CONFIGS[WORKLOAD].seed + 1000 * rank)
+    name = args.workload if args.workload in ("slm", "long") else WORKLOAD
+    w = synth.CONFIGS[name].scaled(seed=synth.CONFIGS[name].seed + 1000 * rank)
     if args.seq_len:
         w = w.scaled(seq_len=args.seq_len, len_lo=max(1, args.seq_len // 4))
+    # the long-sequence configuration goes through the chunked three-step form, four generations at a time
+    chunk_rows = 4 * w.seq_len if name == "long" else w.n_rows
     tok = synth.make_tokens(w)
     T, V, N = w.n_rows, w.vocab, w.n_seq
     esize = 2 if w.dtype == "bf16" else 4
@@ -252,13 +255,17 @@ def run_ours(args):
     def step(ev=None):
         if ev:
             ev[0].record()
-        rb.rapid_pg_stats_chunk(desc, logits, 0, T, targets, mask, ws)
+        for r0 in range(0, T, chunk_rows):
+            n = min(chunk_rows, T - r0)
+            rb.rapid_pg_stats_chunk(desc, logits[r0:r0 + n], r0, n, targets, mask, ws)
         if ev:
             ev[1].record()
         rb.rapid_pg_finalize(desc, behav, rewards, go, loss, token_logp, adv, stats, ws)
         if ev:
             ev[2].record()
-        rb.rapid_pg_dlogits_chunk(desc, logits, dlogits, 0, T, targets, stats, ws)
+        for r0 in range(0, T, chunk_rows):
+            n = min(chunk_rows, T - r0)
+            rb.rapid_pg_dlogits_chunk(desc, logits[r0:r0 + n], dlogits[r0:r0 + n], r0, n, targets, stats, ws)
         if ev:
             ev[3].record()
 
@@ -318,7 +325,7 @@ def run_ours(args):
 
     # ---- end to end through the public call with HOST buffers ------------------------------------
     e2e = None
-    if not args.skip_e2e:
+    if not args.skip_e2e and name == "slm":
         e2e = run_e2e(rb, args, desc, w, logits, tok, behav, dlogits, ws, loss, token_logp, adv, stats,
                       n_tokens, dev, dist)
 
@@ -332,22 +339,24 @@ def run_ours(args):
         for k in ("seconds", "tokens"):
             cpu.pop(k, None)
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "metric": METRIC if name == "slm" else f"PG loss fwd+bwd tokens/sec at V={V} {w.dtype} (chunked form)",
+        "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "prompts": w.n_prompts, "generations_per_prompt": w.group_size,
+        "config": {"workload": name, "chunk_rows": chunk_rows, "prompts": w.n_prompts,
+                   "generations_per_prompt": w.group_size,
                    "padded_len": w.seq_len, "vocab": V, "logits_dtype": w.dtype,
                    "unmasked_tokens_per_gpu": n_tokens, "rows_per_gpu": T,
                    "l2_policy": f"inputs larger than L2 ({T * row_bytes / 1e9:.1f} GB logits per step)",
                    "eta": 2.0, "parallelism": f"dp{world} (by prompt group, no data-path collective)"},
         "clocks": clocks,
         "e2e": e2e,
-        "gpu_launches": 5 * args.steps,
+        "gpu_launches": (2 + 3 * ((T + chunk_rows - 1) // chunk_rows)) * args.steps,
         "roofline": {"bound": "hbm", "kernel": "dlogits_kernel (pass 2)", "achieved": ach_p2,
                      "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": ach_p2 / peak,
                      "frac_of_8TBs_nominal": ach_p2 / 8000.0, "ms_per_launch": p2,
-                     "algorithmic_bytes_per_launch": bytes_p2, "traffic": TRAFFIC_P2_PER_BYTE and
-                     TRAFFIC_P2_PER_BYTE * bytes_p2},
+                     "algorithmic_bytes_per_launch": bytes_p2,
+                     "traffic": (TRAFFIC_P2_PER_BYTE * bytes_p2) if (TRAFFIC_P2_PER_BYTE and name == "slm") else None},
         "roofline_pass1": {"bound": "hbm", "kernel": "row_stats_kernel (pass 1)", "achieved": ach_p1,
                            "peak": peak, "unit": "GB/s", "frac": ach_p1 / peak,
                            "frac_of_8TBs_nominal": ach_p1 / 8000.0, "ms_per_launch": p1,
@@ -695,8 +704,8 @@ def main():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="slm", choices=["slm", "fused", "onpolicy"],
-                    help="slm: the logits-in path the metric is quoted on (default); fused: the LM-head form")
+    ap.add_argument("--workload", default="slm", choices=["slm", "fused", "onpolicy", "long"],
+                    help="slm: the logits-in path the metric is quoted on (default); long: the 64 x 4096 x 32000 fp32 configuration through the chunked form; onpolicy: single pass; fused: the LM-head form")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--skip-e2e", action="store_true", help="leave out the host-buffer leg (profiling)")
     ap.add_argument("--skip-cpu", action="store_true", help="leave out the CPU oracle timing (profiling)")
