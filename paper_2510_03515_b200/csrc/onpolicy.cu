@@ -46,13 +46,19 @@ constexpr int kConsumerWarps = kConsumers / 32;
 constexpr int kThreads = kConsumers + 32;  // + one producer warp
 constexpr int kChunk = RAPID_OP_CHUNK;     // bytes per stage
 constexpr int kStages = RAPID_OP_STAGES;
-constexpr int kMaxPending = 3;             // bulk stores that may still be reading their stage
+#ifndef RAPID_OP_PENDING
+#define RAPID_OP_PENDING 3
+#endif
+constexpr int kMaxPending = RAPID_OP_PENDING;  // bulk stores that may still be reading their stage
 static_assert(kStages >= kMaxPending + 2, "the ring must keep cycling while stores are in flight");
 static_assert((kChunk / 16) % kConsumers == 0, "a chunk is a whole number of 16-byte vectors per consumer");
 constexpr int kVecPerChunk = kChunk / 16;
 constexpr int kVecPerThread = kVecPerChunk / kConsumers;
 constexpr int kVecPerWarp = kVecPerThread * 32;  // a warp's contiguous slice of a chunk, in 16-byte vectors
-constexpr int kZeroBuf = 8192;
+#ifndef RAPID_OP_ZEROBUF
+#define RAPID_OP_ZEROBUF 8192
+#endif
+constexpr int kZeroBuf = RAPID_OP_ZEROBUF;
 constexpr int kPrepThreads = 256;
 
 // L2 cache policies for bulk copies
@@ -221,12 +227,14 @@ struct Acc {
     float m, s0, s1;
 };
 
+template <bool FULL>
 __device__ __forceinline__ void acc_vec(Acc& a, const uint4 (&q)[kVecPerThread], int nvalid, RowConstBf16*) {
     // bf16: chunk maximum with packed max, then one fused multiply-add and one MUFU exponential per element
     uint32_t mx = 0xff80ff80u;  // (-inf, -inf)
 #pragma unroll
     for (int j = 0; j < kVecPerThread; ++j)
-        if (j < nvalid) mx = bf16x2_max(mx, bf16x2_max(bf16x2_max(q[j].x, q[j].y), bf16x2_max(q[j].z, q[j].w)));
+        if (FULL || j < nvalid)
+            mx = bf16x2_max(mx, bf16x2_max(bf16x2_max(q[j].x, q[j].y), bf16x2_max(q[j].z, q[j].w)));
     const float bm = fmaxf(bf16_lo(mx), bf16_hi(mx));
     if (bm > a.m) {
         const float f = ex2_approx((a.m - bm) * kLog2e);
@@ -237,7 +245,7 @@ __device__ __forceinline__ void acc_vec(Acc& a, const uint4 (&q)[kVecPerThread],
     const float nm = -a.m * kLog2e;
 #pragma unroll
     for (int j = 0; j < kVecPerThread; ++j) {
-        if (j < nvalid) {
+        if (FULL || j < nvalid) {
             const uint32_t w[4] = {q[j].x, q[j].y, q[j].z, q[j].w};
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
@@ -247,11 +255,12 @@ __device__ __forceinline__ void acc_vec(Acc& a, const uint4 (&q)[kVecPerThread],
         }
     }
 }
+template <bool FULL>
 __device__ __forceinline__ void acc_vec(Acc& a, const uint4 (&q)[kVecPerThread], int nvalid, RowConstF32*) {
     float bm = -INFINITY;
 #pragma unroll
     for (int j = 0; j < kVecPerThread; ++j)
-        if (j < nvalid)
+        if (FULL || j < nvalid)
             bm = fmaxf(bm, fmaxf(fmaxf(__uint_as_float(q[j].x), __uint_as_float(q[j].y)),
                                  fmaxf(__uint_as_float(q[j].z), __uint_as_float(q[j].w))));
     if (bm > a.m) {
@@ -262,7 +271,7 @@ __device__ __forceinline__ void acc_vec(Acc& a, const uint4 (&q)[kVecPerThread],
     }
 #pragma unroll
     for (int j = 0; j < kVecPerThread; ++j) {
-        if (j < nvalid) {
+        if (FULL || j < nvalid) {
             a.s0 += expf(__uint_as_float(q[j].x) - a.m) + expf(__uint_as_float(q[j].y) - a.m);
             a.s1 += expf(__uint_as_float(q[j].z) - a.m) + expf(__uint_as_float(q[j].w) - a.m);
         }
@@ -278,6 +287,7 @@ __device__ __forceinline__ void acc_scalar(Acc& a, float z, bool base2) {
     a.s0 += base2 ? ex2_approx((z - a.m) * kLog2e) : expf(z - a.m);
 }
 
+template <bool HAS_Y>
 __device__ __forceinline__ uint4 dz_vec(uint4 z, int e0, const RowConstBf16& rc) {
     uint32_t w[4] = {z.x, z.y, z.z, z.w};
 #pragma unroll
@@ -285,7 +295,7 @@ __device__ __forceinline__ uint4 dz_vec(uint4 z, int e0, const RowConstBf16& rc)
         const float lo = ex2_approx(fmaf(bf16_lo(w[k]), kLog2e, rc.c));
         const float hi = ex2_approx(fmaf(bf16_hi(w[k]), kLog2e, rc.c));
         uint32_t out = pack_bf16x2(lo, hi) ^ rc.sign2;
-        if (e0 + 2 * k == (rc.y & ~1)) {  // the sampled token: g (p_y - 1), formed in float
+        if (HAS_Y && e0 + 2 * k == (rc.y & ~1)) {  // the sampled token: g (p_y - 1), formed in float
             const float ps = (rc.y & 1) ? hi : lo;
             const uint32_t b = to_bf16_bits((rc.g < 0.f ? -ps : ps) - rc.g);
             out = (rc.y & 1) ? ((out & 0x0000ffffu) | (b << 16)) : ((out & 0xffff0000u) | b);
@@ -294,13 +304,14 @@ __device__ __forceinline__ uint4 dz_vec(uint4 z, int e0, const RowConstBf16& rc)
     }
     return make_uint4(w[0], w[1], w[2], w[3]);
 }
+template <bool HAS_Y>
 __device__ __forceinline__ uint4 dz_vec(uint4 zb, int e0, const RowConstF32& rc) {
     const float z[4] = {__uint_as_float(zb.x), __uint_as_float(zb.y), __uint_as_float(zb.z), __uint_as_float(zb.w)};
     uint32_t o[4];
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
         float v = rc.g * expf((z[k] - rc.M) - rc.a);
-        if (e0 + k == rc.y) v -= rc.g;
+        if (HAS_Y && e0 + k == rc.y) v -= rc.g;
         o[k] = __float_as_uint(v);
     }
     return make_uint4(o[0], o[1], o[2], o[3]);
@@ -378,6 +389,21 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
     const int n_chunks = (load_bytes + kChunk - 1) / kChunk;
     const int nvec_row = vocab / PER;
     const int whole = nvec_row * 16;  // bytes of a row in whole vectors of real columns
+    // CTA b owns rows b, b + grid, b + 2 grid, ... and walks them starting at a turn proportional to b,
+    // wrapping around: at any moment the CTAs are spread over the whole batch, so the memory system sees
+    // the batch's average mix of rows that are read and written and rows that are only zero-filled
+    // instead of one kind after the other.
+    const int64_t n_turns = (n_rows + gridDim.x - 1) / gridDim.x;
+#ifdef RAPID_OP_NO_ROTATE
+    const int64_t turn0 = 0;
+#else
+    const int64_t turn0 = (n_turns * blockIdx.x) / gridDim.x;
+#endif
+    auto row_of_turn = [&](int64_t k) -> int64_t {
+        int64_t i = turn0 + k;
+        if (i >= n_turns) i -= n_turns;
+        return i * gridDim.x + blockIdx.x;
+    };
 
     if (warp == kConsumerWarps) {
         // ------------------------------- producer -------------------------------------------
@@ -385,15 +411,30 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
             const uint64_t keep = policy_evict_last(), stream = policy_evict_first();
             uint32_t it = 0;
             bool ok = true;
-            for (int64_t r = blockIdx.x; r < n_rows && ok; r += gridDim.x) {
+            for (int64_t k = 0; k < n_turns && ok; ++k) {
+                const int64_t r = row_of_turn(k);
+                if (r >= n_rows) continue;
                 uint8_t st;
                 const int plan = row_plan(r, seq_len, vocab, targets, mask, ws, want_logp != 0, &st);
-                if (plan == ROWS_NONE) continue;
+                if (plan == ROWS_NONE) {
+                    // a row nobody reads gets its zeros from here, ahead of the consumers and outside their
+                    // accounting of pending stores (whole vectors; the consumers write the few columns after them)
+                    uint8_t* orow = static_cast<uint8_t*>(dlogits) + (size_t)r * ld * ESIZE;
+                    for (int o = 0; o < whole; o += kZeroBuf)
+                        bulk_store_hint(orow + o, zeros, (uint32_t)min(kZeroBuf, whole - o), stream);
+                    bulk_commit();
+                    continue;
+                }
                 const uint8_t* src = static_cast<const uint8_t*>(logits) + (size_t)r * ld * ESIZE;
                 for (int sweep = 0; sweep < plan && ok; ++sweep) {
                     // first sweep of a row that will be read again: ask L2 to keep it
                     const uint64_t pol = (sweep == 0 && plan == ROWS_BOTH) ? keep : stream;
-                    for (int c = 0; c < n_chunks; ++c, ++it) {
+                    for (int cc = 0; cc < n_chunks; ++cc, ++it) {
+#ifdef RAPID_OP_REVERSE
+                        const int c = (sweep == 1) ? n_chunks - 1 - cc : cc;  // second sweep: freshest chunks first
+#else
+                        const int c = cc;
+#endif
                         const int s = it % kStages;
                         const uint32_t use = it / kStages;
                         if (use > 0 && !mbar_wait_bounded(&empty_bar[s], (use & 1u) ^ 1u, abortp)) {
@@ -415,12 +456,20 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
                         if (global_timer_ns() - t0 > kWaitLimitNs) break;
                 }
             }
+            bulk_wait_all<0>();  // the zero fills have left the zero buffer
         }
     } else {
         // ------------------------------- consumers ------------------------------------------
         const uint64_t stream = policy_evict_first();
-        uint32_t it = 0;
+        int st = 0;         // stage of the next chunk
+        uint32_t ph = 0;    // and the phase of its barriers
         bool ok = true;
+        auto next_stage = [&]() {
+            if (++st == kStages) {
+                st = 0;
+                ph ^= 1u;
+            }
+        };
         // stages whose outgoing store may still be reading them, newest first (-1: nothing to release);
         // lane 0 of every warp keeps its own (bulk groups belong to the thread that commits them)
         int pend[kMaxPending];
@@ -440,25 +489,31 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
         };
         // give back the oldest outstanding stage, waiting only for that one store
         auto drain_one = [&]() {
-            if (pend[2] != -2) {
-                bulk_wait_read<2>();
-                release(pend[2]);
-                pend[2] = -2;
-            } else if (pend[1] != -2) {
-                bulk_wait_read<1>();
-                release(pend[1]);
-                pend[1] = -2;
-            } else if (pend[0] != -2) {
-                bulk_wait_read<0>();
-                release(pend[0]);
-                pend[0] = -2;
+            bool done = false;
+#pragma unroll
+            for (int i = kMaxPending - 1; i >= 0; --i) {
+                if (!done && pend[i] != -2) {
+                    switch (i) {
+                        case 0: bulk_wait_read<0>(); break;
+                        case 1: bulk_wait_read<1>(); break;
+                        case 2: bulk_wait_read<2>(); break;
+                        case 3: bulk_wait_read<3>(); break;
+                        case 4: bulk_wait_read<4>(); break;
+                        default: bulk_wait_read<5>(); break;
+                    }
+                    release(pend[i]);
+                    pend[i] = -2;
+                    done = true;
+                }
             }
         };
-        static_assert(kMaxPending == 3, "drain_one is written for three pending stores");
+        static_assert(kMaxPending >= 1 && kMaxPending <= 6, "drain_one covers up to six pending stores");
 
         // After a timeout a warp stops working (ok = false) but keeps walking the rows, so that it
         // still meets the others at the next live row's barrier, where all agree to leave.
-        for (int64_t r = blockIdx.x; r < n_rows; r += gridDim.x) {
+        for (int64_t k = 0; k < n_turns; ++k) {
+            const int64_t r = row_of_turn(k);
+            if (r >= n_rows) continue;
             uint8_t state;
             const int plan = row_plan(r, seq_len, vocab, targets, mask, ws, want_logp != 0, &state);
             uint8_t* orow = static_cast<uint8_t*>(dlogits) + (size_t)r * ld * ESIZE;
@@ -475,8 +530,11 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
                     else reinterpret_cast<float*>(orow)[nvec_row * PER + tid - 1] = 0.f;
                 }
             };
-            if (plan == ROWS_NONE) {
-                if (ok) zero_row();
+            if (plan == ROWS_NONE) {  // the producer sends the zeros
+                if (nvec_row * PER + tid < vocab) {
+                    if (ESIZE == 2) reinterpret_cast<uint16_t*>(orow)[nvec_row * PER + tid] = 0;
+                    else reinterpret_cast<float*>(orow)[nvec_row * PER + tid] = 0.f;
+                }
                 if (tid == 0) {
                     ws.row_state[r] = state;
                     ws.lse[r] = 0.0;
@@ -491,24 +549,32 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
             // CTA-wide barrier is needed per chunk ----
             Acc acc{-INFINITY, 0.f, 0.f};
             if (ok) {
-                for (int c = 0; c < n_chunks; ++c, ++it) {
-                    const int s = it % kStages;
-                    const bool got = mbar_wait_bounded(&full_bar[s], (it / kStages) & 1u, abortp);
+                for (int c = 0; c < n_chunks; ++c) {
+                    const int s = st;
+                    const bool got = mbar_wait_bounded(&full_bar[s], ph, abortp);
                     if (__any_sync(0xffffffffu, !got)) {
                         ok = false;
                         break;
                     }
+                    next_stage();
                     const uint4* sv = reinterpret_cast<const uint4*>(ring + (size_t)s * kChunk);
                     const int v0 = c * kVecPerChunk;
                     const int nv = min(kVecPerChunk, nvec_row - v0);
+                    const uint4* wv = sv + warp * kVecPerWarp + lane;  // this thread's vectors: wv[32 j]
+                    const int nvw = nv - warp * kVecPerWarp;           // whole vectors in this warp's slice
+                    const bool full = nvw >= kVecPerWarp;              // the same for the whole warp
                     uint4 q[kVecPerThread];
                     int nvalid = 0;
+                    if (full) {
 #pragma unroll
-                    for (int j = 0; j < kVecPerThread; ++j) {
-                        const int v = warp * kVecPerWarp + j * 32 + lane;
-                        if (v < nv) {
-                            q[j] = sv[v];
-                            nvalid = j + 1;
+                        for (int j = 0; j < kVecPerThread; ++j) q[j] = wv[j * 32];
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < kVecPerThread; ++j) {
+                            if (j * 32 + lane < nvw) {
+                                q[j] = wv[j * 32];
+                                nvalid = j + 1;
+                            }
                         }
                     }
                     float ztail = 0.f;
@@ -532,7 +598,8 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
                         mbar_arrive(&empty_bar[s]);
                         if (c < kMaxPending) drain_one();  // stages still held by this warp's stores of the previous row
                     }
-                    if (nvalid > 0) acc_vec(acc, q, nvalid, (RowConst*)nullptr);
+                    if (full) acc_vec<true>(acc, q, kVecPerThread, (RowConst*)nullptr);
+                    else if (nvalid > 0) acc_vec<false>(acc, q, nvalid, (RowConst*)nullptr);
                     if (has_tail) acc_scalar(acc, ztail, kBase2);
                 }
             }
@@ -550,19 +617,22 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
                     ok = false;
                     break;
                 }
-                if (tid == 0) {
-                    float mm = sh_m[0];
-                    for (int w = 1; w < kConsumerWarps; ++w) mm = fmaxf(mm, sh_m[w]);
-                    double tot = 0.0;
-                    for (int w = 0; w < kConsumerWarps; ++w)
-                        if (sh_s[w] > 0.0) tot += sh_s[w] * exp((double)sh_m[w] - (double)mm);
-                    const double lse = (double)mm + log(tot);
-                    sh_lse = lse;
-                    sh_M = mm;
-                    ws.row_state[r] = ROW_OK;
-                    ws.lse[r] = lse;
-                    ws.token_logp[r] = (double)sh_zy - lse;
-                    ws.row_max[r] = mm;
+                if (warp == 0) {  // one lane per warp's partial: the rescaling exponentials run side by side
+                    const float wmx = lane < kConsumerWarps ? sh_m[lane] : -INFINITY;
+                    const double wsum = lane < kConsumerWarps ? sh_s[lane] : 0.0;
+                    const float mm = warp_max(wmx);
+                    double tot = (wsum > 0.0) ? wsum * exp((double)wmx - (double)mm) : 0.0;
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
+                    if (lane == 0) {
+                        const double lse = (double)mm + log(tot);
+                        sh_lse = lse;
+                        sh_M = mm;
+                        ws.row_state[r] = ROW_OK;
+                        ws.lse[r] = lse;
+                        ws.token_logp[r] = (double)sh_zy - lse;
+                        ws.row_max[r] = mm;
+                    }
                 }
                 consumer_barrier();
             }
@@ -586,13 +656,19 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
                 rc.g = (float)g;
                 rc.y = y;
             }
-            for (int c = 0; c < n_chunks && ok; ++c, ++it) {
-                const int s = it % kStages;
-                const bool got = mbar_wait_bounded(&full_bar[s], (it / kStages) & 1u, abortp);
+            for (int cc = 0; cc < n_chunks && ok; ++cc) {
+#ifdef RAPID_OP_REVERSE
+                const int c = n_chunks - 1 - cc;
+#else
+                const int c = cc;
+#endif
+                const int s = st;
+                const bool got = mbar_wait_bounded(&full_bar[s], ph, abortp);
                 if (__any_sync(0xffffffffu, !got)) {
                     ok = false;
                     break;
                 }
+                next_stage();
                 uint4* sv = reinterpret_cast<uint4*>(ring + (size_t)s * kChunk);
                 const int v0 = c * kVecPerChunk;
                 const int nv = min(kVecPerChunk, nvec_row - v0);
@@ -600,25 +676,32 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
                     const int e = nvec_row * PER + tid;
                     if (e < vocab) dz_scalar(sv, orow, e - v0 * PER, e, rc);
                 }
-                uint4 z[kVecPerThread];
+                uint4* wv = sv + warp * kVecPerWarp + lane;
+                const int nvw = nv - warp * kVecPerWarp;  // whole vectors in this warp's slice
+                const int e0 = (v0 + warp * kVecPerWarp + lane) * PER;  // first column of this thread's first vector
+                if (nvw >= kVecPerWarp) {
+                    uint4 z[kVecPerThread];
 #pragma unroll
-                for (int j = 0; j < kVecPerThread; ++j) {
-                    const int v = warp * kVecPerWarp + j * 32 + lane;
-                    if (v < nv) z[j] = sv[v];
-                }
+                    for (int j = 0; j < kVecPerThread; ++j) z[j] = wv[j * 32];
 #pragma unroll
-                for (int j = 0; j < kVecPerThread; ++j) {
-                    const int v = warp * kVecPerWarp + j * 32 + lane;
-                    if (v < nv) sv[v] = dz_vec(z[j], (v0 + v) * PER, rc);
+                    for (int j = 0; j < kVecPerThread; ++j) {
+                        const int e = e0 + j * 32 * PER;
+                        // the sampled token's column is looked for once per vector, not once per element
+                        wv[j * 32] = ((unsigned)(rc.y - e) < (unsigned)PER) ? dz_vec<true>(z[j], e, rc)
+                                                                            : dz_vec<false>(z[j], e, rc);
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < kVecPerThread; ++j)
+                        if (j * 32 + lane < nvw) wv[j * 32] = dz_vec<true>(wv[j * 32], e0 + j * 32 * PER, rc);
                 }
                 fence_proxy_async_smem();  // generic writes above -> asynchronous read below
                 __syncwarp();
                 if (lane == 0) {
-                    const int nvw = min(kVecPerWarp, nv - warp * kVecPerWarp);  // whole vectors in this warp's slice
                     if (nvw > 0) {
                         const size_t off = (size_t)warp * kVecPerWarp * 16;
                         bulk_store_hint(orow + (size_t)c * kChunk + off, reinterpret_cast<uint8_t*>(sv) + off,
-                                        (uint32_t)nvw * 16u, stream);
+                                        (uint32_t)min(nvw, kVecPerWarp) * 16u, stream);
                         bulk_commit();
                         pushed(s);
                     } else {

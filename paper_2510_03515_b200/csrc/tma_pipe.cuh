@@ -10,6 +10,11 @@
 namespace rapid {
 
 constexpr unsigned long long kWaitLimitNs = 4000000000ull;  // 4 s per wait
+// Upper bound the hardware may keep a waiting thread suspended inside one try_wait before it returns
+// "not yet": long enough that a waiting warp issues next to nothing (waiters would otherwise compete for
+// issue slots with the warps that have work), short against the limit above.  A completed phase wakes
+// the thread at once.
+constexpr uint32_t kSuspendHintNs = 20000u;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -44,10 +49,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(kSuspendHintNs)
         : "memory");
     return ok != 0;
 }
