@@ -590,6 +590,9 @@ def run_onpolicy(args):
     peak, peak_kind = load_peaks()
     row_bytes = V * (2 if w.dtype == "bf16" else 4)
     algo = live_rows * 2 * row_bytes + (T - live_rows) * row_bytes   # live rows: one read + one write
+    # DRAM traffic from the ncu capture summarised under profiles/ (a launch of 8192 rows): reads grow with
+    # the live rows (the second sweep misses L2 for part of each), writes with all rows
+    traffic = TRAFFIC_OP_READ_PER_LIVE_BYTE * live_rows * row_bytes + TRAFFIC_OP_WRITE_PER_ROW_BYTE * T * row_bytes
     ach = algo / (ms_per_step * 1e-3) / 1e9
     line = {
         "metric": "on-policy PG loss fwd+bwd tokens/sec at V=151936 bf16 (single pass)",
@@ -604,7 +607,7 @@ def run_onpolicy(args):
         "clocks": clocks, "e2e": None, "gpu_launches": 4 * args.steps,
         "roofline": {"bound": "hbm", "kernel": "onpolicy_rows_kernel", "achieved": ach, "peak": peak,
                      "peak_kind": peak_kind, "unit": "GB/s", "frac": ach / peak, "frac_of_8TBs_nominal": ach / 8000.0,
-                     "algorithmic_bytes_per_launch": algo, "traffic": None},
+                     "algorithmic_bytes_per_launch": algo, "traffic": traffic},
         "cpu_baseline": None, "stats": {"loss": st["loss"], "status": st["status"]},
     }
     print(json.dumps(line), flush=True)
@@ -615,6 +618,9 @@ def run_onpolicy(args):
 # DRAM traffic of pass 2 per algorithmic byte, from the ncu capture summarised under profiles/
 # (dram__bytes_read.sum + dram__bytes_write.sum of a smaller launch, which scales with rows).
 TRAFFIC_P2_PER_BYTE = 0.9715
+# the on-policy kernel: dram__bytes_read.sum per byte of live rows, dram__bytes_write.sum per byte of all rows
+TRAFFIC_OP_READ_PER_LIVE_BYTE = 1.285
+TRAFFIC_OP_WRITE_PER_ROW_BYTE = 0.976
 
 
 def run_e2e(rb, args, desc, w, logits, tok, behav, dlogits, ws, loss, token_logp, adv, stats,

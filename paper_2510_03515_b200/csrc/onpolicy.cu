@@ -394,11 +394,7 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
     // the batch's average mix of rows that are read and written and rows that are only zero-filled
     // instead of one kind after the other.
     const int64_t n_turns = (n_rows + gridDim.x - 1) / gridDim.x;
-#ifdef RAPID_OP_NO_ROTATE
-    const int64_t turn0 = 0;
-#else
     const int64_t turn0 = (n_turns * blockIdx.x) / gridDim.x;
-#endif
     auto row_of_turn = [&](int64_t k) -> int64_t {
         int64_t i = turn0 + k;
         if (i >= n_turns) i -= n_turns;
@@ -429,12 +425,7 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
                 for (int sweep = 0; sweep < plan && ok; ++sweep) {
                     // first sweep of a row that will be read again: ask L2 to keep it
                     const uint64_t pol = (sweep == 0 && plan == ROWS_BOTH) ? keep : stream;
-                    for (int cc = 0; cc < n_chunks; ++cc, ++it) {
-#ifdef RAPID_OP_REVERSE
-                        const int c = (sweep == 1) ? n_chunks - 1 - cc : cc;  // second sweep: freshest chunks first
-#else
-                        const int c = cc;
-#endif
+                    for (int c = 0; c < n_chunks; ++c, ++it) {
                         const int s = it % kStages;
                         const uint32_t use = it / kStages;
                         if (use > 0 && !mbar_wait_bounded(&empty_bar[s], (use & 1u) ^ 1u, abortp)) {
@@ -656,12 +647,7 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
                 rc.g = (float)g;
                 rc.y = y;
             }
-            for (int cc = 0; cc < n_chunks && ok; ++cc) {
-#ifdef RAPID_OP_REVERSE
-                const int c = n_chunks - 1 - cc;
-#else
-                const int c = cc;
-#endif
+            for (int c = 0; c < n_chunks && ok; ++c) {
                 const int s = st;
                 const bool got = mbar_wait_bounded(&full_bar[s], ph, abortp);
                 if (__any_sync(0xffffffffu, !got)) {
