@@ -395,7 +395,9 @@ def run_fused(args):
         w = w.scaled(seq_len=args.seq_len)
     b = synth.make_head(w, device=dev)
     T, V, D, N = w.n_rows, w.vocab, w.hidden, w.n_seq
-    desc = rb.make_desc(N, w.seq_len, V, w.n_prompts, torch.bfloat16, V, 2.0, 0)
+    stored = args.head == "stored"
+    desc = rb.make_desc(N, w.seq_len, V, w.n_prompts, torch.bfloat16, V, 2.0,
+                        rb.FLAG_HEAD_STORE_LOGITS if stored else 0)
     ws = rb.alloc_fused_head_workspace(desc, D, dev)
     loss = torch.zeros(1, device=dev)
     dh = torch.empty((T, D), dtype=torch.bfloat16, device=dev)
@@ -489,18 +491,22 @@ def run_fused(args):
             dist.destroy_process_group()
         return
     burst, sustained, kind = load_tensor_peaks()
-    flops = 4 * 2.0 * T * D * V   # forward, recompute, dhidden, dW
+    n_gemm = 3 if stored else 4   # forward, (recompute,) dhidden, dW
+    flops = n_gemm * 2.0 * T * D * V
     ach = flops / (ms_per_step * 1e-3) / 1e12
     line = {
         "metric": "fused LM-head PG loss fwd+bwd tokens/sec at V=151936 bf16", "value": tokens / (ms_per_step * 1e-3),
         "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": "fused", "prompts": w.n_prompts, "generations_per_prompt": w.group_size,
+        "config": {"workload": "fused", "head": args.head, "prompts": w.n_prompts, "generations_per_prompt": w.group_size,
                    "padded_len": w.seq_len, "rows_per_gpu": T, "hidden": D, "vocab": V,
                    "l2_policy": "inputs larger than L2 (0.47 GB weight, 5 GB dlogits scratch per step)",
                    "eta": 2.0, "parallelism": f"dp{world} (by prompt group, no data-path collective)"},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": 9 * args.steps,
-        "roofline": {"bound": "tensor", "kernel": "umma gemm_kernel x4 (forward statistics, dlogits, dhidden, dW)",
+        "clocks": clocks, "e2e": e2e, "gpu_launches": (10 if stored else 9) * args.steps,
+        "roofline": {"bound": "tensor",
+                     "kernel": ("umma gemm_kernel x3 (forward statistics + logits store, dhidden, dW); dlogits in place "
+                                "by the logits-in second pass") if stored else
+                               "umma gemm_kernel x4 (forward statistics, dlogits, dhidden, dW)",
                      "achieved": ach, "peak": sustained, "peak_kind": kind + " sustained", "unit": "TFLOP/s",
                      "frac": ach / sustained, "frac_of_burst": ach / burst, "flops_per_step": flops,
                      "traffic": None},
@@ -712,6 +718,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="slm", choices=["slm", "fused", "onpolicy", "long"],
                     help="slm: the logits-in path the metric is quoted on (default); long: the 64 x 4096 x 32000 fp32 configuration through the chunked form; onpolicy: single pass; fused: the LM-head form")
+    ap.add_argument("--head", default="recompute", choices=["recompute", "stored"],
+                    help="--workload fused: form the logits twice on the tensor cores (four contractions), or keep "
+                         "them in bf16 between forward and backward (three contractions)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--skip-e2e", action="store_true", help="leave out the host-buffer leg (profiling)")
     ap.add_argument("--skip-cpu", action="store_true", help="leave out the CPU oracle timing (profiling)")

@@ -79,7 +79,13 @@ enum {
     /* generations (or tokens).  For a mini-batch whose prompt groups are spread over several     */
     /* GPUs: every rank passes the global N (or the global token count), so that the per-rank     */
     /* losses and gradients simply add up to those of the whole mini-batch.                       */
-    RAPID_FLAG_NORM_GIVEN = 32u
+    RAPID_FLAG_NORM_GIVEN = 32u,
+    /* rapid_pg_loss_fused_head only: the forward contraction also writes its logits, rounded to   */
+    /* bf16, into the workspace, and the backward part turns them into dlogits in place instead of */
+    /* forming them a second time on the tensor cores: three GEMM-sized contractions instead of    */
+    /* four, for one more write and read of [T, vocab] bf16.  The row statistics are then those of */
+    /* the rounded logits, i.e. the results are those of rapid_pg_loss_fwd_bwd on bf16(h W).       */
+    RAPID_FLAG_HEAD_STORE_LOGITS = 64u
 };
 
 /* Problem descriptor (host memory, plain data, 48 bytes). */
@@ -316,10 +322,12 @@ rapid_status_t rapid_pg_loss_onpolicy_fwd_bwd(const rapid_desc_t* desc, const vo
  *               holds, besides the per-row state, two floats per row per 256 vocabulary columns
  *               and a bf16 copy of dlogits for at most 16384 rows at a time ([rows, vocab rounded
  *               up to 64 columns]): the backward part runs over the mini-batch in chunks of that
- *               many rows, dW accumulating from chunk to chunk.
+ *               many rows, dW accumulating from chunk to chunk.  With RAPID_FLAG_HEAD_STORE_LOGITS
+ *               the bf16 matrix covers all T rows (it holds the logits first, dlogits afterwards).
  *
  * Tensor-core kernels run for the forward statistics and, per chunk of rows, for dlogits, dhidden
- * and dW (four GEMM-sized contractions over the mini-batch in all), each a persistent grid
+ * and dW (four GEMM-sized contractions over the mini-batch in all; three with
+ * RAPID_FLAG_HEAD_STORE_LOGITS, where dlogits come from the stored logits), each a persistent grid
  * with bounded waits: a wait that gives up raises stats->status to RAPID_ERR_TIMEOUT and leaves the
  * outputs unspecified.  Returns RAPID_ERR_CUDA if the driver cannot encode the tensor maps.
  */

@@ -34,6 +34,7 @@ FLAG_ADV_INPUT_IS_WEIGHT = 4
 FLAG_LEAVE_ONE_OUT = 8
 FLAG_LOO_LITERAL_DIVISOR = 16
 FLAG_NORM_GIVEN = 32
+FLAG_HEAD_STORE_LOGITS = 64
 
 # every symbol declared in include/rapid_pg.h
 EXPORTS = (

@@ -32,7 +32,7 @@ struct HeadScratch {
     float* part_m;   // [n_tiles][T] running maximum of a row within one 256-column tile
     float* part_s;   // [n_tiles][T] sum of exp(z - part_m)
     float* zy;       // [T] the sampled token's logit
-    uint16_t* dz;    // [min(T, kHeadChunkRows)][ldz] bf16
+    uint16_t* dz;    // [min(T, kHeadChunkRows)][ldz] bf16 ([T][ldz] when the logits are stored)
     int* status;     // raised to RAPID_ERR_TIMEOUT by a kernel whose bounded wait ran out
     int64_t ldz;
     int n_tiles;
@@ -53,7 +53,10 @@ inline size_t carve_head(const rapid_desc_t& d, void* base, size_t off0, HeadScr
     s.part_m = reinterpret_cast<float*>(take(nt * T * 4));
     s.part_s = reinterpret_cast<float*>(take(nt * T * 4));
     s.zy = reinterpret_cast<float*>(take(T * 4));
-    s.dz = reinterpret_cast<uint16_t*>(take((T < (size_t)kHeadChunkRows ? T : (size_t)kHeadChunkRows) * ldz * 2));
+    // with stored logits the matrix holds every row's logits first and its dlogits afterwards
+    const bool store_z = (d.flags & RAPID_FLAG_HEAD_STORE_LOGITS) != 0;
+    const size_t dz_rows = (store_z || T < (size_t)kHeadChunkRows) ? T : (size_t)kHeadChunkRows;
+    s.dz = reinterpret_cast<uint16_t*>(take(dz_rows * ldz * 2));
     s.status = reinterpret_cast<int*>(take(256));
     s.ldz = (int64_t)ldz;
     s.n_tiles = (int)nt;
@@ -201,6 +204,84 @@ struct WarpStore {
         if (lane == 0) bulk_wait_all<0>();
         __syncwarp();
     }
+};
+
+// ---- forward epilogue with stored logits: bf16(z) to memory, statistics of the rounded values ----------
+
+struct FwdStatsStore {
+    struct Params {
+        CUtensorMap map;  // z [T, V] bf16, box 64 x 32
+        float* part_m;
+        float* part_s;
+        float* zy;
+        const int32_t* targets;
+        int T, V;
+    };
+    const Params& p;
+    const int quarter, lane;
+    WarpStore st;
+    __device__ FwdStatsStore(const Params& p_, uint8_t* stage, int q, int l) : p(p_), quarter(q), lane(l), st(stage, l) {}
+
+    __device__ void tile(int m0, int n0, uint32_t taddr) {
+        const int row = m0 + quarter * 32 + lane;
+        const int ncols = min(BN, p.V - n0);
+        const int ycol = (row < p.T) ? (p.targets[row] - n0) : -1;
+        float m = -INFINITY, s0 = 0.f, s1 = 0.f, zyv = 0.f;
+#pragma unroll 1
+        for (int q = 0; q * 64 < ncols; ++q) {
+            uint8_t* buf = st.begin();
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const int cc = q * 2 + half;
+                uint32_t r[32];
+                tmem_ld32(taddr + cc * 32, r);
+                tmem_ld_wait();
+                uint32_t o[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) o[j] = pack_bf16x2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    *reinterpret_cast<uint4*>(buf + swz128(lane, half * 4 + k)) =
+                        make_uint4(o[4 * k], o[4 * k + 1], o[4 * k + 2], o[4 * k + 3]);
+                if (cc * 32 >= ncols) continue;  // this half lies beyond the vocabulary
+                // what later steps will read back is the rounded value: the statistics are taken of it
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    r[2 * j] = (cc * 32 + 2 * j < ncols) ? (o[j] << 16) : 0xff800000u;
+                    r[2 * j + 1] = (cc * 32 + 2 * j + 1 < ncols) ? (o[j] & 0xffff0000u) : 0xff800000u;
+                }
+                float cm = __uint_as_float(r[0]);
+#pragma unroll
+                for (int j = 1; j < 32; ++j) cm = fmaxf(cm, __uint_as_float(r[j]));
+                if (cm > m) {
+                    const float f = ex2_approx((m - cm) * kLog2e);
+                    s0 *= f;
+                    s1 *= f;
+                    m = cm;
+                }
+                const float nm = -m * kLog2e;
+#pragma unroll
+                for (int j = 0; j < 32; j += 2) {
+                    s0 += ex2_approx(fmaf(__uint_as_float(r[j]), kLog2e, nm));
+                    s1 += ex2_approx(fmaf(__uint_as_float(r[j + 1]), kLog2e, nm));
+                }
+                if ((ycol >> 5) == cc && ycol >= 0) {
+                    const int jj = ycol & 31;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (j == jj) zyv = __uint_as_float(r[j]);
+                }
+            }
+            st.commit(&p.map, buf, n0 + q * 64, m0 + quarter * 32);
+        }
+        if (row < p.T) {
+            const size_t o = (size_t)(n0 / BN) * (size_t)p.T + (size_t)row;
+            p.part_m[o] = m;
+            p.part_s[o] = s0 + s1;
+            if (ycol >= 0 && ycol < ncols) p.zy[row] = zyv;
+        }
+    }
+    __device__ void finish() { st.finish(); }
 };
 
 // ---- backward epilogue 1: dz in bf16 -------------------------------------------------------------------
@@ -426,11 +507,25 @@ extern "C" rapid_status_t rapid_pg_loss_fused_head(
     clear_status_kernel<<<1, 1, 0, st>>>(hs.status);
 
     // forward
+    const bool store_z = (desc->flags & RAPID_FLAG_HEAD_STORE_LOGITS) != 0;
     {
-        FwdStats::Params fp{hs.part_m, hs.part_s, hs.zy, targets, (int)T, V};
         Shape fwd{(int)((T + BM - 1) / BM), nV, (D + BK - 1) / BK, M_FASTEST};
-        if (launch_gemm<FwdStats, false, true>(h_k, w_mn, fwd, sms, hs.status, fp, st) != cudaSuccess)
-            return RAPID_ERR_CUDA;
+        if (store_z) {
+            FwdStatsStore::Params fp;
+            if (!make_map_bf16(&fp.map, hs.dz, T, V, hs.ldz, 64, 32)) return RAPID_ERR_CUDA;
+            fp.part_m = hs.part_m;
+            fp.part_s = hs.part_s;
+            fp.zy = hs.zy;
+            fp.targets = targets;
+            fp.T = (int)T;
+            fp.V = V;
+            if (launch_gemm<FwdStatsStore, false, true>(h_k, w_mn, fwd, sms, hs.status, fp, st) != cudaSuccess)
+                return RAPID_ERR_CUDA;
+        } else {
+            FwdStats::Params fp{hs.part_m, hs.part_s, hs.zy, targets, (int)T, V};
+            if (launch_gemm<FwdStats, false, true>(h_k, w_mn, fwd, sms, hs.status, fp, st) != cudaSuccess)
+                return RAPID_ERR_CUDA;
+        }
     }
     head_merge_kernel<<<(unsigned)((T + kMergeRows - 1) / kMergeRows), kMergeRows * kMergeSlices, 0, st>>>(
         T, V, hs.n_tiles, hs.part_m, hs.part_s, hs.zy, targets, mask, ws);
@@ -438,21 +533,29 @@ extern "C" rapid_status_t rapid_pg_loss_fused_head(
     if (launch_seq_reduce(*desc, behav_logp, token_logp, ws, st) != cudaSuccess) return RAPID_ERR_CUDA;
     if (launch_finalize(*desc, rewards, group_offsets, loss, adv, stats, ws, st) != cudaSuccess) return RAPID_ERR_CUDA;
 
+    // with stored logits: dlogits in place, by the second pass of the logits-in path
+    if (store_z) {
+        rapid_desc_t dz_desc = *desc;
+        dz_desc.ld = hs.ldz;
+        if (launch_dlogits(dz_desc, hs.dz, hs.dz, 0, T, targets, stats, ws, sms, st) != cudaSuccess) return RAPID_ERR_CUDA;
+    }
+
     // backward, a chunk of rows at a time: dz (recompute), then dh for those rows and the chunk's
     // contribution to dW (the first chunk overwrites dW, later ones add to it, in stream order)
     for (int64_t r0 = 0; r0 < T; r0 += kHeadChunkRows) {
         const int64_t R = (T - r0 < kHeadChunkRows) ? T - r0 : kHeadChunkRows;
         const uint16_t* h_c = static_cast<const uint16_t*>(hidden) + (size_t)r0 * D;
         uint16_t* dh_c = static_cast<uint16_t*>(dhidden) + (size_t)r0 * D;
+        uint16_t* dz_c = hs.dz + (store_z ? (size_t)r0 * (size_t)hs.ldz : 0);  // the chunk's rows of dlogits
         CUtensorMap hc_k, hc_mn, dz_k, dz_mn;
         DzStore::Params dzp;
         StoreBf16::Params dhp;
         StoreF32::Params dwp;
         ok = make_map_bf16(&hc_k, h_c, R, D, D, BK, BM)                // A of recompute: rows x K
              && make_map_bf16(&hc_mn, h_c, R, D, D, 64, BK)            // A of dW: K(=rows) x M(=D)
-             && make_map_bf16(&dz_k, hs.dz, R, V, hs.ldz, BK, BM)      // A of dh: rows x K(=V)
-             && make_map_bf16(&dz_mn, hs.dz, R, V, hs.ldz, 64, BK)     // B of dW: K(=rows) x N(=V)
-             && make_map_bf16(&dzp.map, hs.dz, R, V, hs.ldz, 64, 32)   // stores
+             && make_map_bf16(&dz_k, dz_c, R, V, hs.ldz, BK, BM)      // A of dh: rows x K(=V)
+             && make_map_bf16(&dz_mn, dz_c, R, V, hs.ldz, 64, BK)     // B of dW: K(=rows) x N(=V)
+             && make_map_bf16(&dzp.map, dz_c, R, V, hs.ldz, 64, 32)   // stores
              && make_map_bf16(&dhp.map, dh_c, R, D, D, 64, 32) && make_map_f32(&dwp.map, dW, D, V, ld, 32, 32);
         if (!ok) return RAPID_ERR_CUDA;
         const int mR = (int)((R + BM - 1) / BM);
@@ -467,7 +570,7 @@ extern "C" rapid_status_t rapid_pg_loss_fused_head(
         dzp.seq_len = desc->seq_len;
         dzp.row0 = (int)r0;
         Shape sdz{mR, nV, (D + BK - 1) / BK, M_FASTEST};
-        if (launch_gemm<DzStore, false, true>(hc_k, w_mn, sdz, sms, hs.status, dzp, st) != cudaSuccess)
+        if (!store_z && launch_gemm<DzStore, false, true>(hc_k, w_mn, sdz, sms, hs.status, dzp, st) != cudaSuccess)
             return RAPID_ERR_CUDA;
 
         dhp.N = D;

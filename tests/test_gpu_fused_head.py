@@ -6,6 +6,16 @@ dh and dW: the library rounds dlogits to bf16 before the two products, an indepe
 error of at most 2^-9 per element, so an output element sum_k a_k dz_k carries a random error of
 standard deviation about 2^-9 sqrt(sum_k a_k^2 dz_k^2) / sqrt(3); the test allows 2^-6 times that
 root-sum-square (many standard deviations), plus 2^-8 |ref| for dh's own rounding to bf16.
+
+With RAPID_FLAG_HEAD_STORE_LOGITS the library works on bf16(h W): the oracle then rounds its float64
+logits to bf16 before step 1.  The library rounds a float32 accumulator, the oracle the exact
+product; where the exact logit lies within the accumulator's error (taken as 2^-20 sum_k |h_k W_kv|:
+sixteen float32 ulps of the sum of magnitudes) of a rounding boundary the two may land on
+neighbouring bf16 values.  A token log-probability z_y - lse then moves
+by one bf16 ulp of z_y if the sampled token's logit is such an element, and by p_v ulp(z_v) for every
+other such element v of the row (d lse / d z_v = p_v).  The test computes exactly that bound per row
+from the oracle's own logits and adds it to the usual tolerance; it is far below the tolerance for
+the typical row and matters where a high-probability token sits on a boundary.
 """
 import numpy as np
 import pytest
@@ -23,6 +33,11 @@ def bf16_to_f64(bits):
     return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
 
 
+def round_to_bf16(x):
+    """float64 -> nearest bf16 value, as float64."""
+    return torch.from_numpy(np.ascontiguousarray(x, np.float32)).to(torch.bfloat16).double().numpy()
+
+
 def oracle_head(b, w, eta=2.0, flags=0):
     """Everything the oracle computes for one fused-head batch (small sizes: dense float64)."""
     T, V, L = w.n_rows, w.vocab, w.seq_len
@@ -30,6 +45,18 @@ def oracle_head(b, w, eta=2.0, flags=0):
     tg, mk = b["targets"].numpy(), b["mask"].numpy()
     z = oracle.head_logits(h_bits, w_bits)
     ok = (mk != 0) & (tg >= 0) & (tg < V)
+    logp_slack = np.zeros(T)
+    if flags & rb.FLAG_HEAD_STORE_LOGITS:
+        acc_err = 2.0 ** -20 * (np.abs(bf16_to_f64(h_bits)) @ np.abs(bf16_to_f64(w_bits)))
+        either = np.abs(round_to_bf16(z + acc_err) - round_to_bf16(z - acc_err))   # one ulp where the rounding may go either way
+        z = round_to_bf16(z)
+        prob = np.exp(z - z.max(1, keepdims=True))
+        prob /= prob.sum(1, keepdims=True)
+        rows = np.arange(T)
+        ycol = np.where(ok, tg, 0)
+        prob[rows, ycol] = 1.0                               # the sampled token's own logit counts in full
+        logp_slack = np.where(ok, (prob * either).sum(1), 0.0)
+        flags &= ~rb.FLAG_HEAD_STORE_LOGITS                  # the rest of the oracle does not know the flag
     lse, lp = oracle.token_logp_f64(z, np.where(ok, tg, 0))
     lp = np.where(ok, lp, 0.0)
     behav = b.get("behav_logp")
@@ -44,7 +71,7 @@ def oracle_head(b, w, eta=2.0, flags=0):
     dW = np.zeros((w.hidden, V))
     oracle.head_dweight_accum(dW, dz, h_bits)
     return {"loss": loss, "coef": coef, "seq_logp": S, "token_logp": lp, "adv64": ga["adv64"], "stats": st,
-            "dz": dz, "dh": dh, "dW": dW, "behav": behav, "ok": ok,
+            "dz": dz, "dh": dh, "dW": dW, "behav": behav, "ok": ok, "logp_slack": logp_slack,
             "h": bf16_to_f64(h_bits), "W": bf16_to_f64(w_bits)}
 
 
@@ -80,10 +107,13 @@ def run_head(b, w, behav, ld_pad=0, eta=2.0, flags=0):
 def compare_head(o, g, w):
     dt = torch.bfloat16
     assert g["stats"]["status"] == 0
-    np.testing.assert_allclose(g["token_logp"], o["token_logp"], rtol=0, atol=LOGP_ATOL[dt])
-    np.testing.assert_allclose(g["adv"], o["adv64"], rtol=0, atol=adv_atol(dt, w.seq_len))
+    slack = o["logp_slack"]
+    assert (np.abs(g["token_logp"] - o["token_logp"]) <= LOGP_ATOL[dt] + slack).all()
+    assert np.median(slack) < 5 * LOGP_ATOL[dt], "the relaxation must stay small against the tolerance itself"
+    seq_slack = slack.reshape(w.n_seq, w.seq_len).sum(1).max() * 2.0    # w_n = exp(sum of them), c <= 2
+    np.testing.assert_allclose(g["adv"], o["adv64"], rtol=0, atol=adv_atol(dt, w.seq_len) + seq_slack)
     scale = max(abs(o["loss"]), 1e-3 * float(np.abs(o["coef"] * o["seq_logp"]).sum()), 1e-30)
-    assert abs(g["loss"] - o["loss"]) / scale <= LOSS_RTOL[dt]
+    assert abs(g["loss"] - o["loss"]) / scale <= LOSS_RTOL[dt] + float(np.abs(np.repeat(o["coef"], w.seq_len)) @ slack) / scale
     assert g["stats"]["n_tokens"] == o["stats"]["n_tokens"]
     rss_h = np.sqrt((o["dz"] ** 2) @ (o["W"] ** 2).T)
     tol_h = 2.0 ** -6 * rss_h + 2.0 ** -8 * np.abs(o["dh"]) + 1e-12
@@ -265,3 +295,47 @@ def test_fused_head_shapes_smaller_than_one_tile(V, D, L):
     o = oracle_head(b, w)
     g = run_head(b, w, o["behav"])
     compare_head(o, g, w)
+
+
+@pytest.mark.parametrize("V,D,L,pad", [(1000, 192, 40, 0), (777, 200, 50, 7), (5000, 1536, 33, 8), (40, 8, 3, 0)])
+def test_fused_head_stored_logits(V, D, L, pad):
+    """RAPID_FLAG_HEAD_STORE_LOGITS: three contractions, the logits kept in bf16 between forward and
+    backward.  Same ragged shapes as above; the oracle works on its own bf16 rounding of h W."""
+    pad = (-V) % 8 + pad if (V + pad) % 8 else pad
+    w = synth.CONFIGS["fused"].scaled(n_prompts=3, group_size=4, seq_len=L, vocab=V, hidden=D,
+                                      length_mode="uniform", len_lo=max(1, L // 3), reward_mode="per_prompt_const",
+                                      seed=300 + V)
+    b = synth.make_head(w)
+    o = oracle_head(b, w, flags=rb.FLAG_HEAD_STORE_LOGITS)
+    g = run_head(b, w, o["behav"], ld_pad=pad, flags=rb.FLAG_HEAD_STORE_LOGITS)
+    compare_head(o, g, w)
+
+
+def test_fused_head_stored_logits_more_rows_than_one_backward_chunk():
+    """18000 rows with stored logits: the bf16 matrix covers all rows, dh and dW still run per chunk."""
+    w = synth.CONFIGS["fused"].scaled(n_prompts=3, group_size=3, seq_len=2000, vocab=600, hidden=64,
+                                      length_mode="uniform", len_lo=1500, reward_mode="per_prompt", seed=71)
+    b = synth.make_head(w)
+    b["rewards"] = torch.randn(w.n_seq, generator=torch.Generator().manual_seed(8))
+    o = oracle_head(b, w, flags=rb.FLAG_HEAD_STORE_LOGITS)
+    g = run_head(b, w, o["behav"], flags=rb.FLAG_HEAD_STORE_LOGITS)
+    compare_head(o, g, w)
+
+
+def test_fused_head_stored_logits_bad_tokens_and_flags():
+    """Out-of-range token ids, an empty generation, an empty group, token normalisation and the
+    unclipped outer weight, all with stored logits."""
+    w = synth.CONFIGS["fused"].scaled(n_prompts=2, group_size=3, seq_len=10, vocab=304, hidden=64, seed=5)
+    b = synth.make_head(w)
+    b["targets"][3] = 304
+    b["targets"][17] = -5
+    b["mask"][20:30] = 0
+    b["rewards"] = torch.tensor([1.0, 0.0, 0.5, 0.0, 1.0, 1.0])
+    b["group_offsets"] = torch.tensor([0, 3, 3, 6], dtype=torch.int32)
+    w = w.scaled(n_prompts=3, group_size=2)
+    flags = rb.FLAG_HEAD_STORE_LOGITS | rb.FLAG_NORM_TOKENS | rb.FLAG_OUTER_UNCLIPPED
+    o = oracle_head(b, w, 0.5, flags)
+    g = run_head(b, w, o["behav"], eta=0.5, flags=flags)
+    compare_head(o, g, w)
+    assert g["stats"]["n_bad_token"] == 2 and g["stats"]["n_empty_group"] == 1
+    assert np.all(g["dh"][20:30] == 0.0) and np.all(g["dh"][[3, 17]] == 0.0)
