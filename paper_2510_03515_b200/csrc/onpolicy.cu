@@ -38,6 +38,9 @@ namespace {
 #ifndef RAPID_OP_HINTS
 #define RAPID_OP_HINTS 3  // see policy_evict_last() below; 3 measured best by a small margin
 #endif
+#ifndef RAPID_OP_F32X2
+#define RAPID_OP_F32X2 1  // packed two-float arithmetic in the bf16 sweeps
+#endif
 #ifndef RAPID_OP_MINBLOCKS
 #define RAPID_OP_MINBLOCKS 2
 #endif
@@ -243,6 +246,24 @@ __device__ __forceinline__ void acc_vec(Acc& a, const uint4 (&q)[kVecPerThread],
         a.m = bm;
     }
     const float nm = -a.m * kLog2e;
+#if RAPID_OP_F32X2
+    // a pair at a time: one packed multiply-add and one packed addition per two logits
+    const uint64_t k2 = f32x2(kLog2e, kLog2e), nm2 = f32x2(nm, nm);
+    uint64_t s2 = f32x2(a.s0, a.s1);
+#pragma unroll
+    for (int j = 0; j < kVecPerThread; ++j) {
+        if (FULL || j < nvalid) {
+            const uint32_t w[4] = {q[j].x, q[j].y, q[j].z, q[j].w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                float xl, xh;
+                f32x2_split(f32x2_fma(f32x2(bf16_lo(w[k]), bf16_hi(w[k])), k2, nm2), xl, xh);
+                s2 = f32x2_add(s2, f32x2(ex2_approx(xl), ex2_approx(xh)));
+            }
+        }
+    }
+    f32x2_split(s2, a.s0, a.s1);
+#else
 #pragma unroll
     for (int j = 0; j < kVecPerThread; ++j) {
         if (FULL || j < nvalid) {
@@ -254,6 +275,7 @@ __device__ __forceinline__ void acc_vec(Acc& a, const uint4 (&q)[kVecPerThread],
             }
         }
     }
+#endif
 }
 template <bool FULL>
 __device__ __forceinline__ void acc_vec(Acc& a, const uint4 (&q)[kVecPerThread], int nvalid, RowConstF32*) {
@@ -290,10 +312,19 @@ __device__ __forceinline__ void acc_scalar(Acc& a, float z, bool base2) {
 template <bool HAS_Y>
 __device__ __forceinline__ uint4 dz_vec(uint4 z, int e0, const RowConstBf16& rc) {
     uint32_t w[4] = {z.x, z.y, z.z, z.w};
+#if RAPID_OP_F32X2
+    const uint64_t k2 = f32x2(kLog2e, kLog2e), c2 = f32x2(rc.c, rc.c);
+#endif
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
+#if RAPID_OP_F32X2
+        float xl, xh;
+        f32x2_split(f32x2_fma(f32x2(bf16_lo(w[k]), bf16_hi(w[k])), k2, c2), xl, xh);
+        const float lo = ex2_approx(xl), hi = ex2_approx(xh);
+#else
         const float lo = ex2_approx(fmaf(bf16_lo(w[k]), kLog2e, rc.c));
         const float hi = ex2_approx(fmaf(bf16_hi(w[k]), kLog2e, rc.c));
+#endif
         uint32_t out = pack_bf16x2(lo, hi) ^ rc.sign2;
         if (HAS_Y && e0 + 2 * k == (rc.y & ~1)) {  // the sampled token: g (p_y - 1), formed in float
             const float ps = (rc.y & 1) ? hi : lo;
