@@ -141,7 +141,7 @@ def torch_token_logp(logits: torch.Tensor, targets: torch.Tensor, rows_per_block
 # CPU oracle timing (cpu_baseline leg and --impl reference)
 # ------------------------------------------------------------------------------------------------
 
-def oracle_sample(w: synth.Workload, target_seconds: float = 10.0):
+def oracle_sample(w: synth.Workload, target_seconds: float = 10.0, single_thread: bool = True):
     """Time the oracle, as it stands, on a bounded sample of the workload: whole groups of the
     same vocabulary and dtype with proportionally shorter generations.  Returns a dict."""
     import numpy as np
@@ -175,10 +175,20 @@ def oracle_sample(w: synth.Workload, target_seconds: float = 10.0):
         k = int(min(w.n_prompts, 4, max(1, target_seconds // max(dt, 1e-3))))
         if k > 1:
             dt, ntok, ws = run(seq_len, k)
+    # the same on one thread, on a sample shorter by the core count (one prompt group)
+    single = None
+    if cores > 1 and single_thread:
+        oracle.set_threads(1)
+        try:
+            dt1, ntok1, ws1 = run(max(16, min(ws.seq_len, ws.seq_len * ws.n_prompts // cores)))
+            single = {"value": ntok1 / dt1, "unit": UNIT, "cores": 1,
+                      "sample": f"{ws1.n_seq} generations x {ws1.seq_len} padded tokens ({ntok1} unmasked), {dt1:.2f} s"}
+        finally:
+            oracle.set_threads(cores)
     return {"value": ntok / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"{ws.n_seq} generations x {ws.seq_len} padded tokens ({ntok} unmasked), "
                       f"V={ws.vocab} {ws.dtype}, float64 steps 1-6, {dt:.2f} s",
-            "seconds": dt, "tokens": ntok}
+            "single_thread": single, "seconds": dt, "tokens": ntok}
 
 
 def run_reference(args):
@@ -187,11 +197,11 @@ def run_reference(args):
         return
     w = synth.CONFIGS[WORKLOAD]
     for _ in range(max(0, min(args.warmup, 1))):
-        oracle_sample(w, target_seconds=1.0)
+        oracle_sample(w, target_seconds=1.0, single_thread=False)
     steps = max(1, min(args.steps, 3))
     tot_tok, tot_s, last = 0, 0.0, None
     for _ in range(steps):
-        last = oracle_sample(w, target_seconds=8.0)
+        last = oracle_sample(w, target_seconds=8.0, single_thread=(_ == steps - 1))
         tot_tok += last["tokens"]
         tot_s += last["seconds"]
     value = tot_tok / tot_s
@@ -203,7 +213,7 @@ def run_reference(args):
         "config": {"workload": WORKLOAD + " (bounded sample per step)", "vocab": w.vocab,
                    "logits_dtype": w.dtype},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": last["cores"], "kind": "oracle",
-                         "sample": last["sample"]},
+                         "sample": last["sample"], "single_thread": last["single_thread"]},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
