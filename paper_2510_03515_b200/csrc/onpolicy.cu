@@ -11,10 +11,12 @@
 //   onpolicy_prep_kernel    Eq. 2 advantages, coefficients, token count           (one CTA)
 //   onpolicy_rows_kernel    per live row: sweep 1 streams the row through a shared-memory ring
 //                           (bulk copies) and accumulates max / sum of exponentials; sweep 2 streams
-//                           the same row again -- it was read microseconds ago and is asked to stay
-//                           in L2 (evict-last hint) -- turns it into dlogits in place in shared memory
-//                           and sends it out with bulk stores.  Dead rows (masked, invalid token,
-//                           zero coefficient) are zero-filled from a shared-memory zero buffer.
+//                           the same row again -- it was read microseconds ago and mostly still is
+//                           in L2 (the second read and all stores carry evict-first hints so that
+//                           they do not push it out) -- turns it into dlogits in place in shared
+//                           memory and sends it out with bulk stores.  Dead rows (masked, invalid
+//                           token, zero coefficient) are zero-filled from a shared-memory zero
+//                           buffer, by the producer thread when nobody reads the row.
 //   onpolicy_loss_kernel    S_n = sum_t log pi(y_t), loss = - sum_n g_n S_n, statistics (one CTA)
 //
 // Every wait on a barrier is bounded; a wait that gives up raises RAPID_ERR_TIMEOUT in the
