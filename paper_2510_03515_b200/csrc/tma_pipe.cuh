@@ -2,7 +2,7 @@
 //
 // Every wait is bounded: a waiter polls the barrier and, after a wall-clock limit, raises a
 // CTA-wide abort flag and gives up, so that a fault elsewhere can never leave a kernel spinning.
-// Copies are never multicast and never cross to another GPU.
+// Every copy has one destination, this CTA's shared memory, and none crosses to another GPU.
 #pragma once
 
 #include <stdint.h>

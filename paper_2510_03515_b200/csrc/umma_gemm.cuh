@@ -12,7 +12,7 @@
 //   * the epilogue is a functor; it reads the accumulator with tcgen05.ld and does whatever the
 //     caller needs (row statistics, dlogits, plain stores)
 //
-// No multicast, no clusters, nothing crosses to another GPU.  Every wait is bounded: on a timeout
+// One CTA per tile and one destination per copy (no clusters); nothing crosses to another GPU.  Every wait is bounded: on a timeout
 // the CTA raises an abort flag, all roles leave their loops, outstanding copies and MMAs are given
 // a bounded time to land, tensor memory is freed and *status is raised to RAPID_ERR_TIMEOUT.
 #pragma once
