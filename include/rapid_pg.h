@@ -165,7 +165,9 @@ rapid_status_t rapid_group_advantage(const rapid_desc_t* desc, const float* rewa
  *                 (in place).  Partial overlap is not allowed.  Rows that are masked, or whose
  *                 coefficient g_n is zero, are written as zeros.  Columns >= vocab are untouched.
  *   loss          [1] float out
- *   token_logp    [T] float out (0 on masked rows); may be NULL
+ *   token_logp    [T] float out (0 on masked rows); may be NULL.  token_logp[r] - behav_logp[r] is
+ *                 the token-level importance weight in log scale that Sec. 4.3 plots for a single
+ *                 generation; stats->n_clipped / N is the clipped share it reports per inner step
  *   adv           [N] float out; may be NULL
  *   stats         out; may be NULL
  *   workspace     rapid_workspace_bytes(desc) bytes, 256-byte aligned
