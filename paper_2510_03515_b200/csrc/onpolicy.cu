@@ -247,7 +247,7 @@ __device__ __forceinline__ void acc_vec(Acc& a, const uint4 (&q)[kVecPerThread],
         a.s1 *= f;
         a.m = bm;
     }
-    const float nm = -a.m * kLog2e;
+    const float nm = (a.m == -INFINITY) ? 0.f : -a.m * kLog2e;  // all -inf so far: no (-inf) - (-inf)
 #if RAPID_OP_F32X2
     // a pair at a time: one packed multiply-add and one packed addition per two logits
     const uint64_t k2 = f32x2(kLog2e, kLog2e), nm2 = f32x2(nm, nm);
@@ -293,6 +293,7 @@ __device__ __forceinline__ void acc_vec(Acc& a, const uint4 (&q)[kVecPerThread],
         a.s1 *= f;
         a.m = bm;
     }
+    if (a.m == -INFINITY) return;  // nothing but -inf so far: the sums stay 0
 #pragma unroll
     for (int j = 0; j < kVecPerThread; ++j) {
         if (FULL || j < nvalid) {
@@ -302,6 +303,7 @@ __device__ __forceinline__ void acc_vec(Acc& a, const uint4 (&q)[kVecPerThread],
     }
 }
 __device__ __forceinline__ void acc_scalar(Acc& a, float z, bool base2) {
+    if (z == -INFINITY) return;  // contributes nothing
     if (z > a.m) {
         const float f = base2 ? ex2_approx((a.m - z) * kLog2e) : expf(a.m - z);
         a.s0 *= f;

@@ -57,7 +57,9 @@ __device__ __forceinline__ void bf16_batch(const uint4 (&q)[U], float& m, FloatS
         S.scale(ex2_approx((m - bm) * kLog2e));
         m = bm;
     }
-    const float nm = -m * kLog2e;
+    // logits may be -inf (a masked part of the vocabulary): while the thread has seen nothing else its
+    // maximum is -inf too, and the shift must not turn (-inf) - (-inf) into a NaN
+    const float nm = (m == -INFINITY) ? 0.f : -m * kLog2e;
     float s0 = 0.f, s1 = 0.f;
 #pragma unroll
     for (int j = 0; j < U; ++j) {
@@ -117,7 +119,7 @@ __device__ __forceinline__ void row_sweep_bf16(const uint16_t* row, int vocab, f
             S.scale(ex2_approx((m - z) * kLog2e));
             m = z;
         }
-        tail = (double)ex2_approx((z - m) * kLog2e);
+        if (z != -INFINITY) tail = (double)ex2_approx((z - m) * kLog2e);
     }
     m_out = m;
     s_out = S.value() + tail;
@@ -136,6 +138,7 @@ __device__ __forceinline__ void f32_batch(const float4* q, int n, float& m, doub
         if (s > 0.0) s *= exp((double)m - (double)bm);
         m = bm;
     }
+    if (m == -INFINITY) return;  // nothing but -inf so far (a masked part of the vocabulary): the sum stays 0
     for (int j = 0; j < n; ++j)
         s += (double)((expf(q[j].x - m) + expf(q[j].y - m)) + (expf(q[j].z - m) + expf(q[j].w - m)));
 }
@@ -174,7 +177,7 @@ __device__ __forceinline__ void row_sweep_f32(const float* row, int vocab, float
             if (s > 0.0) s *= exp((double)m - (double)z);
             m = z;
         }
-        s += (double)expf(z - m);
+        if (z != -INFINITY) s += (double)expf(z - m);
     }
     m_out = m;
     s_out = s;

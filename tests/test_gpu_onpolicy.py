@@ -199,3 +199,27 @@ def test_slm_config_full_size():
         blk = logits[r0:r0 + 4096].float()
         assert torch.isfinite(blk).all() and (blk[~live[r0:r0 + 4096]] == 0).all()
         assert blk.sum(1).abs().max().item() <= 1e-3
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_minus_infinity_logits(dtype):
+    """-inf logits (a masked part of the vocabulary): a padded tail on every row, the whole first 9000
+    columns of every third row, a scattered 30 % of every fifth row; never the sampled token."""
+    V = 20000 + (4 if dtype == "f32" else 0)
+    w = synth.Workload("ninf", 2, 3, 7, V, dtype, 2.0, 4.0, "uniform", len_lo=3, behav_sigma=0.3,
+                       reward_mode="per_prompt", seed=812)
+    b = synth.make_batch(w)
+    b["rewards"] = torch.randn(w.n_seq, generator=torch.Generator().manual_seed(3))
+    z = b["logits"]
+    T = z.shape[0]
+    ninf = torch.zeros(z.shape, dtype=torch.bool)
+    ninf[:, V - 613:] = True
+    ninf[0::3, :9000] = True
+    ninf[1::5] |= torch.rand((len(range(1, T, 5)), V), generator=torch.Generator().manual_seed(77)) < 0.3
+    ninf[torch.arange(T), b["targets"].long().clamp(0, V - 1)] = False
+    z[ninf] = float("-inf")
+    o = oracle_onpolicy(b, w.n_seq, w.seq_len, V)
+    g = run_gpu(b, w.n_seq, w.seq_len)
+    compare(o, g, torch.float32 if dtype == "f32" else torch.bfloat16, w.seq_len)
+    assert np.isfinite(g["dlogits"]).all() and np.isfinite(g["token_logp"]).all()
+    assert np.all(g["dlogits"][ninf.numpy()] == 0.0)

@@ -431,3 +431,36 @@ def test_logits_read_from_pinned_host_memory(dtype):
     assert L.rapid_pg_loss_fwd_bwd_hostlogits(*args(pageable.data_ptr())) == rb.RAPID_ERR_INVALID_ARG
     assert L.rapid_pg_loss_fwd_bwd_hostlogits(*args(staging.data_ptr())) == rb.RAPID_ERR_INVALID_ARG
     torch.cuda.synchronize()
+
+
+def _with_minus_infinity(b, V):
+    """Masks parts of the vocabulary with -inf, never the sampled token: a padded tail on every row
+    (as a model whose vocabulary is padded to a round size produces), the whole first 9000 columns of
+    every third row (every thread's first loads see nothing but -inf there), and a scattered 30 % of
+    every fifth row."""
+    z = b["logits"]
+    T = z.shape[0]
+    ninf = torch.zeros(z.shape, dtype=torch.bool)
+    ninf[:, V - 613:] = True
+    ninf[0::3, :9000] = True
+    g = torch.Generator().manual_seed(1234)
+    ninf[1::5] |= torch.rand((len(range(1, T, 5)), V), generator=g) < 0.3
+    ninf[torch.arange(T), b["targets"].long().clamp(0, V - 1)] = False
+    z[ninf] = float("-inf")
+    return ninf
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_minus_infinity_logits(dtype):
+    """-inf logits (a masked part of the vocabulary) contribute exp(-inf) = 0 to every sum and get a zero
+    gradient; long runs of them at the start of a row must not poison the running maximum."""
+    V = 20000 + (4 if dtype == "f32" else 0)
+    w = synth.Workload("ninf", 2, 3, 7, V, dtype, 2.0, 4.0, "uniform", len_lo=3, behav_sigma=0.3,
+                       reward_mode="per_prompt", seed=811)
+    b = synth.make_batch(w)
+    b["rewards"] = torch.randn(w.n_seq, generator=torch.Generator().manual_seed(3))
+    ninf = _with_minus_infinity(b, V)
+    o, g = run_both(b, w.n_seq, w.seq_len)
+    compare(o, g, _dt(w), w.seq_len)
+    assert np.isfinite(g["dlogits"]).all() and np.isfinite(g["token_logp"]).all()
+    assert np.all(g["dlogits"][ninf.numpy()] == 0.0)

@@ -52,6 +52,31 @@ def test_lse_two_logit_closed_form(oracle):
     assert o["token_logp"][1] == pytest.approx(-math.log1p(math.exp(a - b)), abs=1e-15)
 
 
+@pytest.mark.parametrize("as_bf16", [False, True])
+def test_lse_with_minus_infinity_logits_closed_form(oracle, as_bf16):
+    """A masked part of the vocabulary (-inf logits): with k finite logits all equal to c and the rest -inf,
+    lse = c + ln k, log pi = -ln k on the finite ones, and the gradient is exactly 0 on the masked ones
+    and g (1/k - 1[v = y]) elsewhere."""
+    V, k, c = 64, 5, 1.5
+    z = np.full((3, V), -np.inf, np.float32)
+    cols = [[0, 1, 2, 3, 4], [59, 60, 61, 62, 63], [7, 20, 33, 46, 63]]
+    for r in range(3):
+        z[r, cols[r]] = c
+    y = np.array([2, 63, 33], np.int32)
+    bits = torch.from_numpy(z).to(torch.bfloat16).view(torch.int16).numpy().view("uint16") if as_bf16 else z
+    o = oracle.token_logp(bits, V, y)
+    np.testing.assert_allclose(o["lse"], c + LN(k), rtol=0, atol=1e-15)
+    np.testing.assert_allclose(o["token_logp"], -LN(k), rtol=0, atol=1e-15)
+    g = np.array([0.25, -0.5, 2.0])
+    dz = oracle.dlogits_rows(bits, V, 1, y, o["row_ok"], o["lse"], g, np.arange(3, dtype=np.int64))
+    for r in range(3):
+        ref = np.zeros(V)
+        ref[cols[r]] = g[r] / k
+        ref[y[r]] -= g[r]
+        np.testing.assert_allclose(dz[r], ref, rtol=0, atol=1e-15)
+        assert np.all(dz[r][np.isinf(z[r])] == 0.0)
+
+
 def test_lse_brute_force_fsum(oracle):
     """Naive log(sum(exp z)) with an exactly rounded sum (math.fsum) on tiny rows."""
     rng = np.random.default_rng(5)
