@@ -155,8 +155,8 @@ rapid_status_t rapid_group_advantage(const rapid_desc_t* desc, const float* rewa
  * re-read pass that writes dlogits).
  *   logits        [T, ld] of desc->dtype, row-major; only the first `vocab` entries of a row
  *                 are used.  Base address and ld * sizeof(element) must be multiples of 16.
- *                 Entries may be -inf (a masked part of the vocabulary: probability and gradient
- *                 exactly 0) as long as the sampled token's and at least one other entry of every
+ *                 Entries may be -inf or the dtype's lowest finite value (a masked part of the
+ *                 vocabulary: probability and gradient exactly 0) as long as the sampled token's and at least one other entry of every
  *                 unmasked row is finite; +inf and NaN are not accepted (results unspecified).
  *   targets       [T] int32, the sampled token y_r
  *   mask          [T] uint8, non-zero = the token counts; NULL = all ones.  Masked rows of

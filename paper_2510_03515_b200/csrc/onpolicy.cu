@@ -247,7 +247,8 @@ __device__ __forceinline__ void acc_vec(Acc& a, const uint4 (&q)[kVecPerThread],
         a.s1 *= f;
         a.m = bm;
     }
-    const float nm = (a.m == -INFINITY) ? 0.f : -a.m * kLog2e;  // all -inf so far: no (-inf) - (-inf)
+    // nothing but -inf (or the lowest finite value) so far: no (-inf) - (-inf), no overflow of the shift
+    const float nm = (a.m < -1.0e38f) ? 0.f : -a.m * kLog2e;
 #if RAPID_OP_F32X2
     // a pair at a time: one packed multiply-add and one packed addition per two logits
     const uint64_t k2 = f32x2(kLog2e, kLog2e), nm2 = f32x2(nm, nm);

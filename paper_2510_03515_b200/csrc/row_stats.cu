@@ -57,9 +57,10 @@ __device__ __forceinline__ void bf16_batch(const uint4 (&q)[U], float& m, FloatS
         S.scale(ex2_approx((m - bm) * kLog2e));
         m = bm;
     }
-    // logits may be -inf (a masked part of the vocabulary): while the thread has seen nothing else its
-    // maximum is -inf too, and the shift must not turn (-inf) - (-inf) into a NaN
-    const float nm = (m == -INFINITY) ? 0.f : -m * kLog2e;
+    // logits may be -inf or the lowest finite value (a masked part of the vocabulary): while the thread
+    // has seen nothing else its maximum is that too, and the shift -m log2(e) must neither turn
+    // (-inf) - (-inf) into a NaN nor overflow to +inf
+    const float nm = (m < -1.0e38f) ? 0.f : -m * kLog2e;
     float s0 = 0.f, s1 = 0.f;
 #pragma unroll
     for (int j = 0; j < U; ++j) {

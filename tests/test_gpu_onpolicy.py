@@ -201,8 +201,9 @@ def test_slm_config_full_size():
         assert blk.sum(1).abs().max().item() <= 1e-3
 
 
+@pytest.mark.parametrize("fill", ["-inf", "lowest"])
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-def test_minus_infinity_logits(dtype):
+def test_minus_infinity_logits(dtype, fill):
     """-inf logits (a masked part of the vocabulary): a padded tail on every row, the whole first 9000
     columns of every third row, a scattered 30 % of every fifth row; never the sampled token."""
     V = 20000 + (4 if dtype == "f32" else 0)
@@ -217,7 +218,7 @@ def test_minus_infinity_logits(dtype):
     ninf[0::3, :9000] = True
     ninf[1::5] |= torch.rand((len(range(1, T, 5)), V), generator=torch.Generator().manual_seed(77)) < 0.3
     ninf[torch.arange(T), b["targets"].long().clamp(0, V - 1)] = False
-    z[ninf] = float("-inf")
+    z[ninf] = float("-inf") if fill == "-inf" else torch.finfo(z.dtype).min
     o = oracle_onpolicy(b, w.n_seq, w.seq_len, V)
     g = run_gpu(b, w.n_seq, w.seq_len)
     compare(o, g, torch.float32 if dtype == "f32" else torch.bfloat16, w.seq_len)

@@ -433,7 +433,7 @@ def test_logits_read_from_pinned_host_memory(dtype):
     torch.cuda.synchronize()
 
 
-def _with_minus_infinity(b, V):
+def _with_minus_infinity(b, V, fill="-inf"):
     """Masks parts of the vocabulary with -inf, never the sampled token: a padded tail on every row
     (as a model whose vocabulary is padded to a round size produces), the whole first 9000 columns of
     every third row (every thread's first loads see nothing but -inf there), and a scattered 30 % of
@@ -446,12 +446,14 @@ def _with_minus_infinity(b, V):
     g = torch.Generator().manual_seed(1234)
     ninf[1::5] |= torch.rand((len(range(1, T, 5)), V), generator=g) < 0.3
     ninf[torch.arange(T), b["targets"].long().clamp(0, V - 1)] = False
-    z[ninf] = float("-inf")
+    # "lowest": the most negative finite value of the dtype, which some pipelines use as their mask value
+    z[ninf] = float("-inf") if fill == "-inf" else torch.finfo(z.dtype).min
     return ninf
 
 
+@pytest.mark.parametrize("fill", ["-inf", "lowest"])
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-def test_minus_infinity_logits(dtype):
+def test_minus_infinity_logits(dtype, fill):
     """-inf logits (a masked part of the vocabulary) contribute exp(-inf) = 0 to every sum and get a zero
     gradient; long runs of them at the start of a row must not poison the running maximum."""
     V = 20000 + (4 if dtype == "f32" else 0)
@@ -459,7 +461,7 @@ def test_minus_infinity_logits(dtype):
                        reward_mode="per_prompt", seed=811)
     b = synth.make_batch(w)
     b["rewards"] = torch.randn(w.n_seq, generator=torch.Generator().manual_seed(3))
-    ninf = _with_minus_infinity(b, V)
+    ninf = _with_minus_infinity(b, V, fill)
     o, g = run_both(b, w.n_seq, w.seq_len)
     compare(o, g, _dt(w), w.seq_len)
     assert np.isfinite(g["dlogits"]).all() and np.isfinite(g["token_logp"]).all()
