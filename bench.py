@@ -5,11 +5,18 @@ A "step" is one pass of the whole path (row statistics, finalize, dlogits) over 
 mini-batch of the SLM shape: 8 prompts x 8 generations, responses of 256-1024 tokens padded to
 1024 and masked, V = 151936, bf16 logits.  The metric is unmasked tokens per second.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload ...]
 
-N > 1 is launched with torch.distributed.run, one rank per GPU; every rank runs its own
-mini-batch (the path partitions by prompt group, so there is no collective on the data path:
-weak scaling) and the time is the maximum over ranks.
+N ranks, one per GPU: either start this file under torch.distributed.run (WORLD_SIZE etc. in the
+environment), or give --gpus N > 1 to a plain `python bench.py`, which then starts
+`python -m torch.distributed.run --nnodes=1 --nproc-per-node N --master-addr 127.0.0.1 ...` on
+itself after checking that the machine has N devices (it refuses otherwise).  Every rank runs
+its own mini-batch (the path partitions by prompt group, so there is no collective on the data
+path: weak scaling); the time is the maximum over ranks, the tokens the sum.
+
+The default single-GPU run appends short timed runs of the other forms of the path to the same
+JSON line (`roofline_onpolicy`, `roofline_fused`, `roofline_fused_stored`, `roofline_long`),
+each with its own clock record; --no-extras leaves them out.
 
 --impl reference times the float64 CPU oracle, as it stands, on the host cores (the paper ships
 no implementation to run); each of its steps is a bounded sample of the same workload.
@@ -221,23 +228,133 @@ def run_reference(args):
 
 
 # ------------------------------------------------------------------------------------------------
-# the CUDA path
+# ranks, launching, timing
 # ------------------------------------------------------------------------------------------------
 
-def run_ours(args):
-    from paper_2510_03515_b200 import binding as rb
+def launch_command(gpus: int, env: dict, argv: list, device_count: int, port: int):
+    """What a plain `python bench.py --gpus N` has to do.  Returns
+       ("run", None)     this process is the (or a) rank: go on;
+       ("exec", [cmd])   start N ranks with torch.distributed.run on this file;
+       ("error", text)   the request cannot be met (too few devices, or ranks that contradict --gpus)."""
+    if "WORLD_SIZE" in env:
+        world = int(env["WORLD_SIZE"])
+        if gpus != world:
+            return "error", f"--gpus {gpus} but the launcher started WORLD_SIZE={world} ranks"
+        return "run", None
+    if gpus <= 1:
+        return "run", None
+    if device_count < gpus:
+        return "error", (f"--gpus {gpus} asked for, but this machine has {device_count} CUDA device(s): "
+                         f"refusing to print a line for fewer ranks than asked")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+    return "exec", cmd
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
+
+def free_port() -> int:
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        return sk.getsockname()[1]
+
+
+class Rank:
+    """This process's place among the ranks; the NCCL group carries only timings and token counts."""
+
+    def __init__(self):
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+        if self.local_rank >= torch.cuda.device_count():
+            raise SystemExit(f"rank {self.rank}: no CUDA device {self.local_rank} "
+                             f"({torch.cuda.device_count()} on this machine)")
+        torch.cuda.set_device(self.local_rank)
+        self.dev = torch.device("cuda", self.local_rank)
+        self.dist = None
+        if self.world > 1:
+            import torch.distributed as dist
+            if not dist.is_initialized():
+                dist.init_process_group("nccl", device_id=self.dev)
+            self.dist = dist
+
+    def barrier(self):
+        if self.dist:
+            self.dist.barrier()
+
+    def max_over_ranks(self, x: float) -> float:
+        if not self.dist:
+            return float(x)
+        t = torch.tensor([x], device=self.dev, dtype=torch.float64)
+        self.dist.all_reduce(t, op=self.dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def sum_over_ranks(self, x: float) -> float:
+        if not self.dist:
+            return float(x)
+        t = torch.tensor([x], device=self.dev, dtype=torch.float64)
+        self.dist.all_reduce(t, op=self.dist.ReduceOp.SUM)
+        return float(t.item())
+
+    def close(self):
+        if self.dist and self.dist.is_initialized():
+            self.dist.destroy_process_group()
+
+
+def timed_region(rk: Rank, step, steps: int, n_marks: int):
+    """Barrier + synchronize, `steps` calls of step(events), synchronize + barrier.  `step` records
+    its `n_marks` events (first = start of the step, last = its end) on the current stream, which is
+    the stream the library launches on.  Returns (total ms, maximum over ranks; per-step lists of
+    the n_marks - 1 intervals in ms, this rank's; the clock record taken meanwhile)."""
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(n_marks)] for _ in range(steps)]
+    sampler = ClockSampler(rk.local_rank) if rk.rank == 0 else None
+    rk.barrier()
+    torch.cuda.synchronize()
+    if sampler:
+        sampler.start()
+        time.sleep(0.25)
+    t0w = time.time()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for k in range(steps):
+        step(evs[k])
+    end.record()
+    torch.cuda.synchronize()
+    t1w = time.time()
+    rk.barrier()
+    clocks = sampler.stop(t0w, t1w) if sampler else None
+    total_ms = rk.max_over_ranks(start.elapsed_time(end))
+    parts = [[e[i].elapsed_time(e[i + 1]) for e in evs] for i in range(n_marks - 1)]
+    whole = [e[0].elapsed_time(e[-1]) for e in evs]
+    return total_ms, parts, whole, clocks
+
+
+def mean_median(xs):
+    return statistics.mean(xs), statistics.median(xs)
+
+
+# ------------------------------------------------------------------------------------------------
+# the logits-in path (--workload slm, the metric's configuration; --workload long, chunked form)
+# ------------------------------------------------------------------------------------------------
+
+# DRAM traffic per algorithmic byte, from the ncu captures summarised under profiles/ (counters
+# dram__bytes_read.sum + dram__bytes_write.sum of a smaller launch of the same kernel; traffic grows
+# in proportion to the rows processed).  NOT counters of this run: the line says so.
+TRAFFIC_P2_PER_BYTE = 0.9715
+TRAFFIC_P2_SOURCE = "profiles/logits_in_path_slm_bf16.md: ncu dram bytes of a 2.5 GB launch x rows of this one"
+# the on-policy kernel: dram__bytes_read.sum per byte of live rows, dram__bytes_write.sum per byte of all rows
+TRAFFIC_OP_READ_PER_LIVE_BYTE = 1.285
+TRAFFIC_OP_WRITE_PER_ROW_BYTE = 0.976
+TRAFFIC_OP_SOURCE = "profiles/onpolicy_rows_kernel_slm_bf16.md: ncu dram bytes of an 8192-row launch x rows of this one"
+# pass 1's secondary ceiling: share of cycles the MUFU (ex2) pipe is busy, same captures
+MUFU_PIPE_PCT_PASS1 = 70.0
+MUFU_SOURCE = "profiles/logits_in_path_slm_bf16.md (ncu pipe utilisation of row_stats_kernel)"
+
+
+def run_ours(args, rk: Rank):
+    from paper_2510_03515_b200 import binding as rb
+    rank, dev, world = rk.rank, rk.dev, rk.world
     rb.lib()
 
     name = args.workload if args.workload in ("slm", "long") else WORKLOAD
@@ -283,46 +400,17 @@ def run_ours(args):
         step()
     torch.cuda.synchronize()
     st = rb.read_stats(stats)
-    live_rows = None
     # rows pass 2 really streams: unmasked rows of generations with a non-zero coefficient
     coef_live = (adv != 0).repeat_interleave(w.seq_len)
     live_rows = int((coef_live & (mask != 0)).sum().item())
 
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
-    sampler = ClockSampler(local_rank) if rank == 0 else None
-    if dist:
-        dist.barrier()
-    torch.cuda.synchronize()
-    if sampler:
-        sampler.start()
-        time.sleep(0.25)
-    t0w = time.time()
-    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    start.record()
-    for k in range(args.steps):
-        step(evs[k])
-    end.record()
-    torch.cuda.synchronize()
-    t1w = time.time()
-    if dist:
-        dist.barrier()
-    clocks = sampler.stop(t0w, t1w) if sampler else None
-    elapsed_ms = start.elapsed_time(end)
-    if dist:
-        t = torch.tensor([elapsed_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
-        tk = torch.tensor([n_tokens], device=dev, dtype=torch.float64)
-        dist.all_reduce(tk, op=dist.ReduceOp.SUM)
-        total_tokens = float(tk.item())
-    else:
-        total_tokens = float(n_tokens)
+    elapsed_ms, parts, whole, clocks = timed_region(rk, step, args.steps, 4)
+    total_tokens = rk.sum_over_ranks(n_tokens)
     ms_per_step = elapsed_ms / args.steps
     value = total_tokens / (ms_per_step * 1e-3)
+    ms_median = rk.max_over_ranks(statistics.median(whole))
 
-    p1 = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)
-    fin = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)
-    p2 = statistics.mean(e[2].elapsed_time(e[3]) for e in evs)
+    (p1, p1_med), (fin, _), (p2, p2_med) = (mean_median(x) for x in parts)
     peak, peak_kind = load_peaks()
     row_bytes = V * esize
     # algorithmic bytes: pass 1 reads every unmasked row once; pass 2 re-reads the live rows and
@@ -334,25 +422,25 @@ def run_ours(args):
     ach_all = (bytes_p1 + bytes_p2) / (ms_per_step * 1e-3) / 1e9
 
     # ---- end to end through the public call with HOST buffers ------------------------------------
-    e2e = None
+    e2e = e2e_grad = None
     if not args.skip_e2e and name == "slm":
-        e2e = run_e2e(rb, args, desc, w, logits, tok, behav, dlogits, ws, loss, token_logp, adv, stats,
-                      n_tokens, dev, dist)
+        e2e, e2e_grad = run_e2e(rb, args, desc, w, logits, tok, behav, dlogits, ws, loss, token_logp, adv, stats,
+                                n_tokens, rk)
 
     if rank != 0:
-        if dist:
-            dist.destroy_process_group()
-        return
+        return None
     cpu = None
     if not args.skip_cpu:
-        cpu = oracle_sample(w, target_seconds=10.0)
+        cpu = oracle_sample(w, target_seconds=args.cpu_seconds)
         for k in ("seconds", "tokens"):
             cpu.pop(k, None)
+    n_chunks = (T + chunk_rows - 1) // chunk_rows
     line = {
         "metric": METRIC if name == "slm" else f"PG loss fwd+bwd tokens/sec at V={V} {w.dtype} (chunked form)",
         "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "ms_per_step_median": ms_median, "value_at_median": total_tokens / (ms_median * 1e-3),
         "config": {"workload": name, "chunk_rows": chunk_rows, "prompts": w.n_prompts,
                    "generations_per_prompt": w.group_size,
                    "padded_len": w.seq_len, "vocab": V, "logits_dtype": w.dtype,
@@ -361,290 +449,44 @@ def run_ours(args):
                    "eta": 2.0, "parallelism": f"dp{world} (by prompt group, no data-path collective)"},
         "clocks": clocks,
         "e2e": e2e,
-        "gpu_launches": (2 + 3 * ((T + chunk_rows - 1) // chunk_rows)) * args.steps,
+        "e2e_gradient_to_host": e2e_grad,
+        "gpu_launches": (2 + 3 * n_chunks) * args.steps,
         "roofline": {"bound": "hbm", "kernel": "dlogits_kernel (pass 2)", "achieved": ach_p2,
                      "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": ach_p2 / peak,
-                     "frac_of_8TBs_nominal": ach_p2 / 8000.0, "ms_per_launch": p2,
-                     "algorithmic_bytes_per_launch": bytes_p2,
-                     "traffic": (TRAFFIC_P2_PER_BYTE * bytes_p2) if (TRAFFIC_P2_PER_BYTE and name == "slm") else None},
+                     "frac_of_8TBs_nominal": ach_p2 / 8000.0, "ms_per_launch": p2 / n_chunks,
+                     "ms_per_step": p2, "ms_per_step_median": p2_med,
+                     "achieved_at_median": bytes_p2 / (p2_med * 1e-3) / 1e9,
+                     "algorithmic_bytes_per_launch": bytes_p2 / n_chunks, "launches_per_step": 2 * n_chunks,
+                     "traffic": (TRAFFIC_P2_PER_BYTE * bytes_p2) if name == "slm" else None,
+                     "traffic_source": TRAFFIC_P2_SOURCE if name == "slm" else None},
         "roofline_pass1": {"bound": "hbm", "kernel": "row_stats_kernel (pass 1)", "achieved": ach_p1,
                            "peak": peak, "unit": "GB/s", "frac": ach_p1 / peak,
-                           "frac_of_8TBs_nominal": ach_p1 / 8000.0, "ms_per_launch": p1,
-                           "algorithmic_bytes_per_launch": bytes_p1},
+                           "frac_of_8TBs_nominal": ach_p1 / 8000.0, "ms_per_launch": p1 / n_chunks,
+                           "ms_per_step": p1, "ms_per_step_median": p1_med,
+                           "achieved_at_median": bytes_p1 / (p1_med * 1e-3) / 1e9,
+                           "algorithmic_bytes_per_launch": bytes_p1 / n_chunks, "launches_per_step": n_chunks,
+                           "secondary_ceiling": {"pipe": "MUFU ex2", "pipe_active_pct": MUFU_PIPE_PCT_PASS1,
+                                                 "source": MUFU_SOURCE} if w.dtype == "bf16" else None},
         "roofline_step": {"achieved": ach_all, "peak": peak, "unit": "GB/s", "frac": ach_all / peak,
                           "frac_of_8TBs_nominal": ach_all / 8000.0, "finalize_ms": fin},
         "cpu_baseline": cpu,
         "stats": {"n_clipped": st["n_clipped"], "mean_log_cw": st["mean_log_cw"], "loss": st["loss"]},
     }
-    print(json.dumps(line), flush=True)
-    if dist:
-        dist.destroy_process_group()
+    return line
 
 
-# ------------------------------------------------------------------------------------------------
-# the fused LM-head form (--workload fused): hidden states and the LM-head weight in, no logits
-# ------------------------------------------------------------------------------------------------
-
-def run_fused(args):
-    from paper_2510_03515_b200 import binding as rb
-
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
-    rb.lib()
-    w = synth.CONFIGS["fused"].scaled(seed=synth.CONFIGS["fused"].seed + 1000 * rank)
-    if args.seq_len:
-        w = w.scaled(seq_len=args.seq_len)
-    b = synth.make_head(w, device=dev)
-    T, V, D, N = w.n_rows, w.vocab, w.hidden, w.n_seq
-    stored = args.head == "stored"
-    desc = rb.make_desc(N, w.seq_len, V, w.n_prompts, torch.bfloat16, V, 2.0,
-                        rb.FLAG_HEAD_STORE_LOGITS if stored else 0)
-    ws = rb.alloc_fused_head_workspace(desc, D, dev)
-    loss = torch.zeros(1, device=dev)
-    dh = torch.empty((T, D), dtype=torch.bfloat16, device=dev)
-    dW = torch.empty((D, V), dtype=torch.float32, device=dev)
-    tl = torch.empty(T, device=dev)
-    adv = torch.empty(N, device=dev)
-    stats = rb.alloc_stats(dev)
-    behav = torch.full((T,), -12.0, device=dev)
-
-    def step(hid=None, wv=None, bh=None):
-        rb.rapid_pg_loss_fused_head(desc, b["hidden"] if hid is None else hid, b["w_vocab"] if wv is None else wv,
-                                    b["targets"], b["mask"], behav if bh is None else bh, b["rewards"],
-                                    b["group_offsets"], loss, dh, dW, tl, adv, stats, ws)
-
-    step()   # the library's own token log-probs seed the synthetic behaviour log-probs (input synthesis)
-    torch.cuda.synchronize()
-    behav = (tl + b["behav_noise"]).contiguous()
-    for _ in range(args.warmup):
-        step()
-    torch.cuda.synchronize()
-    sampler = ClockSampler(local_rank) if rank == 0 else None
-    if dist:
-        dist.barrier()
-    torch.cuda.synchronize()
-    if sampler:
-        sampler.start()
-        time.sleep(0.25)
-    t0w = time.time()
-    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    start.record()
-    for _ in range(args.steps):
-        step()
-    end.record()
-    torch.cuda.synchronize()
-    t1w = time.time()
-    if dist:
-        dist.barrier()
-    clocks = sampler.stop(t0w, t1w) if sampler else None
-    ms = start.elapsed_time(end)
-    n_tokens = int(b["mask"].sum().item())
-    tokens = float(n_tokens)
-    if dist:
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-        tk = torch.tensor([tokens], device=dev, dtype=torch.float64)
-        dist.all_reduce(tk, op=dist.ReduceOp.SUM)
-        tokens = float(tk.item())
-    ms_per_step = ms / args.steps
-    st = rb.read_stats(stats)
-
-    # end to end: hidden states, weight and per-token arrays start in pinned host memory
-    e2e = None
-    if not args.skip_e2e:
-        names = ("hidden", "w_vocab")
-        host = {k: b[k].cpu().pin_memory() for k in names}
-        h_behav = behav.cpu().pin_memory()
-        d_in = {k: torch.empty_like(b[k]) for k in names}
-        d_behav = torch.empty_like(behav)
-        h_loss = torch.empty(1, dtype=torch.float32).pin_memory()
-        h2d = sum(v.numel() * v.element_size() for v in host.values()) + h_behav.numel() * 4
-
-        def e2e_step():
-            for k in names:
-                d_in[k].copy_(host[k], non_blocking=True)
-            d_behav.copy_(h_behav, non_blocking=True)
-            step(d_in["hidden"], d_in["w_vocab"], d_behav)
-            h_loss.copy_(loss, non_blocking=True)
-            torch.cuda.current_stream().synchronize()
-
-        e2e_step()
-        if dist:
-            dist.barrier()
-        torch.cuda.synchronize()
-        k = max(1, min(args.e2e_steps, args.steps))
-        s2, e2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        s2.record()
-        for _ in range(k):
-            e2e_step()
-        e2.record()
-        torch.cuda.synchronize()
-        ems = s2.elapsed_time(e2)
-        if dist:
-            t = torch.tensor([ems], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ems = float(t.item())
-        e2e = {"value": tokens * k / (ems * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
-               "d2h_bytes_per_step": 4, "steps": k, "ms_per_step": ems / k}
-    if rank != 0:
-        if dist:
-            dist.destroy_process_group()
-        return
-    burst, sustained, kind = load_tensor_peaks()
-    n_gemm = 3 if stored else 4   # forward, (recompute,) dhidden, dW
-    flops = n_gemm * 2.0 * T * D * V
-    ach = flops / (ms_per_step * 1e-3) / 1e12
-    line = {
-        "metric": "fused LM-head PG loss fwd+bwd tokens/sec at V=151936 bf16", "value": tokens / (ms_per_step * 1e-3),
-        "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": "fused", "head": args.head, "prompts": w.n_prompts, "generations_per_prompt": w.group_size,
-                   "padded_len": w.seq_len, "rows_per_gpu": T, "hidden": D, "vocab": V,
-                   "l2_policy": "inputs larger than L2 (0.47 GB weight, 5 GB dlogits scratch per step)",
-                   "eta": 2.0, "parallelism": f"dp{world} (by prompt group, no data-path collective)"},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": (10 if stored else 9) * args.steps,
-        "roofline": {"bound": "tensor",
-                     "kernel": ("umma gemm_kernel x3 (forward statistics + logits store, dhidden, dW); dlogits in place "
-                                "by the logits-in second pass") if stored else
-                               "umma gemm_kernel x4 (forward statistics, dlogits, dhidden, dW)",
-                     "achieved": ach, "peak": sustained, "peak_kind": kind + " sustained", "unit": "TFLOP/s",
-                     "frac": ach / sustained, "frac_of_burst": ach / burst, "flops_per_step": flops,
-                     "traffic": None},
-        "cpu_baseline": None,
-        "stats": {"n_clipped": st["n_clipped"], "mean_log_cw": st["mean_log_cw"], "loss": st["loss"],
-                  "status": st["status"]},
-    }
-    print(json.dumps(line), flush=True)
-    if dist:
-        dist.destroy_process_group()
-
-
-# ------------------------------------------------------------------------------------------------
-# the on-policy single-pass form (--workload onpolicy): same mini-batch as slm, weights all one
-# ------------------------------------------------------------------------------------------------
-
-def run_onpolicy(args):
-    from paper_2510_03515_b200 import binding as rb
-
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
-    w = synth.CONFIGS["slm"].scaled(seed=synth.CONFIGS["slm"].seed + 1000 * rank)
-    if args.seq_len:
-        w = w.scaled(seq_len=args.seq_len, len_lo=max(1, args.seq_len // 4))
-    tok = synth.make_tokens(w)
-    T, V, N = w.n_rows, w.vocab, w.n_seq
-    logits = synth.logits_for_sequences(w, tok["targets"], 0, N, device=dev)
-    targets, mask = tok["targets"].to(dev), tok["mask"].to(dev)
-    rewards, go = tok["rewards"].to(dev), tok["group_offsets"].to(dev)
-    dlogits = torch.empty_like(logits)
-    desc = rb.make_desc(N, w.seq_len, V, w.n_prompts, logits.dtype, logits.stride(0), 2.0, 0)
-    ws = rb.alloc_workspace(desc, dev)
-    loss = torch.zeros(1, device=dev)
-    adv = torch.empty(N, device=dev)
-    stats = rb.alloc_stats(dev)
-    n_tokens = int(tok["mask"].sum().item())
-
-    def step():
-        rb.rapid_pg_loss_onpolicy_fwd_bwd(desc, logits, targets, mask, rewards, go, dlogits, loss, None, adv, stats, ws)
-
-    for _ in range(args.warmup):
-        step()
-    torch.cuda.synchronize()
-    live_rows = int(((adv != 0).repeat_interleave(w.seq_len) & (mask != 0)).sum().item())
-    sampler = ClockSampler(local_rank) if rank == 0 else None
-    if dist:
-        dist.barrier()
-    torch.cuda.synchronize()
-    if sampler:
-        sampler.start()
-        time.sleep(0.25)
-    t0w = time.time()
-    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    start.record()
-    for _ in range(args.steps):
-        step()
-    end.record()
-    torch.cuda.synchronize()
-    t1w = time.time()
-    if dist:
-        dist.barrier()
-    clocks = sampler.stop(t0w, t1w) if sampler else None
-    ms = start.elapsed_time(end)
-    tokens = float(n_tokens)
-    if dist:
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-        tk = torch.tensor([tokens], device=dev, dtype=torch.float64)
-        dist.all_reduce(tk, op=dist.ReduceOp.SUM)
-        tokens = float(tk.item())
-    if rank != 0:
-        if dist:
-            dist.destroy_process_group()
-        return
-    ms_per_step = ms / args.steps
-    st = rb.read_stats(stats)
-    peak, peak_kind = load_peaks()
-    row_bytes = V * (2 if w.dtype == "bf16" else 4)
-    algo = live_rows * 2 * row_bytes + (T - live_rows) * row_bytes   # live rows: one read + one write
-    # DRAM traffic from the ncu capture summarised under profiles/ (a launch of 8192 rows): reads grow with
-    # the live rows (the second sweep misses L2 for part of each), writes with all rows
-    traffic = TRAFFIC_OP_READ_PER_LIVE_BYTE * live_rows * row_bytes + TRAFFIC_OP_WRITE_PER_ROW_BYTE * T * row_bytes
-    ach = algo / (ms_per_step * 1e-3) / 1e9
-    line = {
-        "metric": "on-policy PG loss fwd+bwd tokens/sec at V=151936 bf16 (single pass)",
-        "value": tokens / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": "onpolicy (slm mini-batch, mu = pi_theta)", "prompts": w.n_prompts,
-                   "generations_per_prompt": w.group_size, "padded_len": w.seq_len, "vocab": V,
-                   "logits_dtype": w.dtype, "unmasked_tokens_per_gpu": n_tokens, "live_rows_per_gpu": live_rows,
-                   "rows_per_gpu": T, "l2_policy": "inputs larger than L2",
-                   "parallelism": f"dp{world} (by prompt group, no data-path collective)"},
-        "clocks": clocks, "e2e": None, "gpu_launches": 4 * args.steps,
-        "roofline": {"bound": "hbm", "kernel": "onpolicy_rows_kernel", "achieved": ach, "peak": peak,
-                     "peak_kind": peak_kind, "unit": "GB/s", "frac": ach / peak, "frac_of_8TBs_nominal": ach / 8000.0,
-                     "algorithmic_bytes_per_launch": algo, "traffic": traffic},
-        "cpu_baseline": None, "stats": {"loss": st["loss"], "status": st["status"]},
-    }
-    print(json.dumps(line), flush=True)
-    if dist:
-        dist.destroy_process_group()
-
-
-# DRAM traffic of pass 2 per algorithmic byte, from the ncu capture summarised under profiles/
-# (dram__bytes_read.sum + dram__bytes_write.sum of a smaller launch, which scales with rows).
-TRAFFIC_P2_PER_BYTE = 0.9715
-# the on-policy kernel: dram__bytes_read.sum per byte of live rows, dram__bytes_write.sum per byte of all rows
-TRAFFIC_OP_READ_PER_LIVE_BYTE = 1.285
-TRAFFIC_OP_WRITE_PER_ROW_BYTE = 0.976
-
-
-def run_e2e(rb, args, desc, w, logits, tok, behav, dlogits, ws, loss, token_logp, adv, stats,
-            n_tokens, dev, dist):
+def run_e2e(rb, args, desc, w, logits, tok, behav, dlogits, ws, loss, token_logp, adv, stats, n_tokens, rk: Rank):
     """Same step, but the inputs start in pinned HOST memory and the loss is read back to the host
     every step.  Uses a full pinned copy of the logits when the host has room, otherwise a
-    2 GiB pinned buffer copied repeatedly into successive device slices (same bytes moved)."""
+    2 GiB pinned buffer copied repeatedly into successive device slices (same bytes moved).
+
+    Two figures.  `e2e`: inputs in, loss out; dlogits, the path's main output, stays in device
+    memory, where the transformer's backward pass consumes it (the method alternates inference and
+    training on the same GPUs, so nothing downstream wants the gradient on the host).
+    `e2e_gradient_to_host`: the same plus a copy of all of dlogits to pinned host memory, for a
+    caller that does want it there; only taken when the host has room for the second buffer."""
     import psutil
+    dev = rk.dev
     T = logits.shape[0]
     nbytes = logits.numel() * logits.element_size()
     steps = max(1, min(args.e2e_steps, args.steps))
@@ -668,13 +510,13 @@ def run_e2e(rb, args, desc, w, logits, tok, behav, dlogits, ws, loss, token_logp
     d_logits = torch.empty_like(logits)
     h_loss = torch.empty(1, dtype=torch.float32).pin_memory()
     h2d = nbytes + sum(v.numel() * v.element_size() for v in small.values()) + h_behav.numel() * 4
-    d2h = 4
 
     direct = host_logits.shape[0] == T   # the whole batch is pinned: let the kernels read it from there
     if direct:
         mode = "full pinned copy, read in place by the statistics pass (masked rows never cross the bus)"
         h2d = n_tokens * logits.shape[1] * logits.element_size() + \
             sum(v.numel() * v.element_size() for v in small.values()) + h_behav.numel() * 4
+    host_grad = None
 
     def step():
         for k in small:
@@ -692,32 +534,302 @@ def run_e2e(rb, args, desc, w, logits, tok, behav, dlogits, ws, loss, token_logp
             rb.rapid_pg_loss_fwd_bwd(desc, d_logits, d["targets"], d["mask"], d_behav, d["rewards"],
                                      d["group_offsets"], dlogits, loss, token_logp, adv, stats, ws)
         h_loss.copy_(loss, non_blocking=True)
+        if host_grad is not None:
+            host_grad.copy_(dlogits, non_blocking=True)
         torch.cuda.current_stream().synchronize()
         return float(h_loss[0])
 
-    step()
-    if dist:
-        dist.barrier()
-    torch.cuda.synchronize()
-    s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    s.record()
-    for _ in range(steps):
+    def timed():
         step()
-    e.record()
+        rk.barrier()
+        torch.cuda.synchronize()
+        s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s.record()
+        for _ in range(steps):
+            step()
+        e.record()
+        torch.cuda.synchronize()
+        return rk.max_over_ranks(s.elapsed_time(e))
+
+    ms = timed()
+    tokens = rk.sum_over_ranks(n_tokens)
+    out = {"value": tokens * steps / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+           "d2h_bytes_per_step": 4, "steps": steps, "ms_per_step": ms / steps, "host_buffer": mode,
+           "d2h_is": "the loss", "result_left_on_device_bytes": int(nbytes),
+           "result_left_on_device": "dlogits (consumed on the device by the backward pass of the model)"}
+    out_grad = None
+    try:
+        enough = psutil.virtual_memory().available > 2 * nbytes
+        enough = bool(rk.sum_over_ranks(0.0 if enough else 1.0) == 0.0)      # every rank, or none
+        if enough:
+            host_grad = torch.empty(logits.shape, dtype=logits.dtype, pin_memory=True)
+            ms2 = timed()
+            out_grad = {"value": tokens * steps / (ms2 * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+                        "d2h_bytes_per_step": int(nbytes) + 4, "steps": steps, "ms_per_step": ms2 / steps,
+                        "d2h_is": "the loss and all of dlogits"}
+    except RuntimeError as ex:          # pinning the second buffer failed: report why, keep the first figure
+        out_grad = {"unavailable": str(ex).splitlines()[0][:200]}
+    del d_logits, host_logits, host_grad
+    return out, out_grad
+
+
+# ------------------------------------------------------------------------------------------------
+# the fused LM-head form (--workload fused): hidden states and the LM-head weight in, no logits
+# ------------------------------------------------------------------------------------------------
+
+def run_fused(args, rk: Rank):
+    from paper_2510_03515_b200 import binding as rb
+    rank, dev, world = rk.rank, rk.dev, rk.world
+    rb.lib()
+    w = synth.CONFIGS["fused"].scaled(seed=synth.CONFIGS["fused"].seed + 1000 * rank)
+    if args.seq_len:
+        w = w.scaled(seq_len=args.seq_len)
+    b = synth.make_head(w, device=dev)
+    T, V, D, N = w.n_rows, w.vocab, w.hidden, w.n_seq
+    stored = args.head == "stored"
+    desc = rb.make_desc(N, w.seq_len, V, w.n_prompts, torch.bfloat16, V, 2.0,
+                        rb.FLAG_HEAD_STORE_LOGITS if stored else 0)
+    ws = rb.alloc_fused_head_workspace(desc, D, dev)
+    loss = torch.zeros(1, device=dev)
+    dh = torch.empty((T, D), dtype=torch.bfloat16, device=dev)
+    dW = torch.empty((D, V), dtype=torch.float32, device=dev)
+    tl = torch.empty(T, device=dev)
+    adv = torch.empty(N, device=dev)
+    stats = rb.alloc_stats(dev)
+    behav = torch.full((T,), -12.0, device=dev)
+
+    def step(ev=None, hid=None, wv=None, bh=None):
+        if ev:
+            ev[0].record()
+        rb.rapid_pg_loss_fused_head(desc, b["hidden"] if hid is None else hid, b["w_vocab"] if wv is None else wv,
+                                    b["targets"], b["mask"], behav if bh is None else bh, b["rewards"],
+                                    b["group_offsets"], loss, dh, dW, tl, adv, stats, ws)
+        if ev:
+            ev[1].record()
+
+    step()   # the library's own token log-probs seed the synthetic behaviour log-probs (input synthesis)
     torch.cuda.synchronize()
-    ms = s.elapsed_time(e)
-    tokens = float(n_tokens)
-    if dist:
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-        tk = torch.tensor([tokens], device=dev, dtype=torch.float64)
-        dist.all_reduce(tk, op=dist.ReduceOp.SUM)
-        tokens = float(tk.item())
-    del d_logits, host_logits
-    return {"value": tokens * steps / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
-            "d2h_bytes_per_step": int(d2h), "steps": steps, "ms_per_step": ms / steps,
-            "host_buffer": mode}
+    behav = (tl + b["behav_noise"]).contiguous()
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    ms, _, whole, clocks = timed_region(rk, step, args.steps, 2)
+    n_tokens = int(b["mask"].sum().item())
+    tokens = rk.sum_over_ranks(n_tokens)
+    ms_per_step = ms / args.steps
+    ms_median = rk.max_over_ranks(statistics.median(whole))
+    st = rb.read_stats(stats)
+
+    # end to end: hidden states, weight and per-token arrays start in pinned host memory
+    e2e = None
+    if not args.skip_e2e:
+        names = ("hidden", "w_vocab")
+        host = {k: b[k].cpu().pin_memory() for k in names}
+        h_behav = behav.cpu().pin_memory()
+        d_in = {k: torch.empty_like(b[k]) for k in names}
+        d_behav = torch.empty_like(behav)
+        h_loss = torch.empty(1, dtype=torch.float32).pin_memory()
+        h2d = sum(v.numel() * v.element_size() for v in host.values()) + h_behav.numel() * 4
+
+        def e2e_step():
+            for k in names:
+                d_in[k].copy_(host[k], non_blocking=True)
+            d_behav.copy_(h_behav, non_blocking=True)
+            step(None, d_in["hidden"], d_in["w_vocab"], d_behav)
+            h_loss.copy_(loss, non_blocking=True)
+            torch.cuda.current_stream().synchronize()
+
+        e2e_step()
+        rk.barrier()
+        torch.cuda.synchronize()
+        k = max(1, min(args.e2e_steps, args.steps))
+        s2, e2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s2.record()
+        for _ in range(k):
+            e2e_step()
+        e2.record()
+        torch.cuda.synchronize()
+        ems = rk.max_over_ranks(s2.elapsed_time(e2))
+        e2e = {"value": tokens * k / (ems * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+               "d2h_bytes_per_step": 4, "steps": k, "ms_per_step": ems / k, "d2h_is": "the loss",
+               "result_left_on_device_bytes": int(dh.numel() * 2 + dW.numel() * 4),
+               "result_left_on_device": "dhidden and dW (consumed on the device by the model's backward pass and optimizer)"}
+    if rank != 0:
+        return None
+    cpu = None
+    if not args.skip_cpu:
+        cpu = oracle_head_sample(w, target_seconds=args.cpu_seconds)
+    burst, sustained, kind = load_tensor_peaks()
+    n_gemm = 3 if stored else 4   # forward, (recompute,) dhidden, dW
+    flops = n_gemm * 2.0 * T * D * V
+    ach = flops / (ms_per_step * 1e-3) / 1e12
+    mhz = (clocks or {}).get("sm_mhz")
+    line = {
+        "metric": "fused LM-head PG loss fwd+bwd tokens/sec at V=151936 bf16", "value": tokens / (ms_per_step * 1e-3),
+        "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "ms_per_step_median": ms_median,
+        "config": {"workload": "fused", "head": args.head, "prompts": w.n_prompts, "generations_per_prompt": w.group_size,
+                   "padded_len": w.seq_len, "rows_per_gpu": T, "hidden": D, "vocab": V,
+                   "l2_policy": "inputs larger than L2 (0.47 GB weight, 5 GB dlogits scratch per step)",
+                   "eta": 2.0, "parallelism": f"dp{world} (by prompt group, no data-path collective)"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": (10 if stored else 9) * args.steps,
+        "roofline": {"bound": "tensor",
+                     "kernel": ("umma gemm_kernel x3 (forward statistics + logits store, dhidden, dW); dlogits in place "
+                                "by the logits-in second pass") if stored else
+                               "umma gemm_kernel x4 (forward statistics, dlogits, dhidden, dW)",
+                     "achieved": ach, "peak": sustained, "peak_kind": kind + " sustained", "unit": "TFLOP/s",
+                     "frac": ach / sustained, "frac_of_burst": ach / burst, "flops_per_step": flops,
+                     "ms_x_sm_mhz": (ms_per_step * mhz) if mhz else None,
+                     "traffic": None},
+        "cpu_baseline": cpu,
+        "stats": {"n_clipped": st["n_clipped"], "mean_log_cw": st["mean_log_cw"], "loss": st["loss"],
+                  "status": st["status"]},
+    }
+    return line
+
+
+def oracle_head_sample(w: synth.Workload, target_seconds: float = 6.0):
+    """The oracle's fused-head steps (float64 product by plain loops, steps 1-6, dhidden, dW), as they
+    stand, on a bounded sample: a few generations of the same hidden size and vocabulary."""
+    import numpy as np
+
+    import oracle
+    cores = oracle.max_threads()
+
+    def run(n_rows):
+        L = max(1, n_rows // 2)
+        ws_ = w.scaled(n_prompts=1, group_size=2, seq_len=L)
+        b = synth.make_head(ws_)
+        hb, wb = synth.bits_numpy(b["hidden"]), synth.bits_numpy(b["w_vocab"])
+        tg = b["targets"].numpy()
+        t0 = time.perf_counter()
+        z = oracle.head_logits(hb, wb)
+        lse, lp = oracle.token_logp_f64(z, tg)
+        behav = (lp + b["behav_noise"].numpy()).astype(np.float32)
+        s_, S_, cnt = oracle.seq_reduce(ws_.n_seq, L, lp, behav, np.ones(ws_.n_rows, np.uint8))
+        ga = oracle.group_advantage(b["rewards"].numpy(), s_, b["group_offsets"].numpy(), 2.0, 0)
+        _, coef, _ = oracle.coef_loss(s_, S_, cnt, ga["weight"], ga["clipped_w"], ga["adv64"], 2.0, 0)
+        dz = oracle.dlogits_f64_inplace(z, tg, lse, np.repeat(coef, L))
+        oracle.head_dhidden(dz, wb)
+        dW = np.zeros((ws_.hidden, ws_.vocab))
+        oracle.head_dweight_accum(dW, dz, hb)
+        return time.perf_counter() - t0, ws_.n_rows
+
+    dt, n = run(8)
+    rows = int(max(8, min(512, 8 * target_seconds / max(dt, 1e-3)))) // 2 * 2
+    if rows > n:
+        dt, n = run(rows)
+    return {"value": n / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{n} rows of hidden size {w.hidden}, V={w.vocab}, float64 product by plain loops, "
+                      f"steps 1-6, dhidden and dW, {dt:.2f} s"}
+
+
+# ------------------------------------------------------------------------------------------------
+# the on-policy single-pass form (--workload onpolicy): same mini-batch as slm, weights all one
+# ------------------------------------------------------------------------------------------------
+
+def run_onpolicy(args, rk: Rank):
+    from paper_2510_03515_b200 import binding as rb
+    rank, dev, world = rk.rank, rk.dev, rk.world
+    w = synth.CONFIGS["slm"].scaled(seed=synth.CONFIGS["slm"].seed + 1000 * rank)
+    if args.seq_len:
+        w = w.scaled(seq_len=args.seq_len, len_lo=max(1, args.seq_len // 4))
+    tok = synth.make_tokens(w)
+    T, V, N = w.n_rows, w.vocab, w.n_seq
+    logits = synth.logits_for_sequences(w, tok["targets"], 0, N, device=dev)
+    targets, mask = tok["targets"].to(dev), tok["mask"].to(dev)
+    rewards, go = tok["rewards"].to(dev), tok["group_offsets"].to(dev)
+    dlogits = torch.empty_like(logits)
+    desc = rb.make_desc(N, w.seq_len, V, w.n_prompts, logits.dtype, logits.stride(0), 2.0, 0)
+    ws = rb.alloc_workspace(desc, dev)
+    loss = torch.zeros(1, device=dev)
+    adv = torch.empty(N, device=dev)
+    stats = rb.alloc_stats(dev)
+    n_tokens = int(tok["mask"].sum().item())
+
+    def step(ev=None):
+        if ev:
+            ev[0].record()
+        rb.rapid_pg_loss_onpolicy_fwd_bwd(desc, logits, targets, mask, rewards, go, dlogits, loss, None, adv, stats, ws)
+        if ev:
+            ev[1].record()
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    live_rows = int(((adv != 0).repeat_interleave(w.seq_len) & (mask != 0)).sum().item())
+    ms, _, whole, clocks = timed_region(rk, step, args.steps, 2)
+    tokens = rk.sum_over_ranks(n_tokens)
+    ms_median = rk.max_over_ranks(statistics.median(whole))
+    if rank != 0:
+        return None
+    ms_per_step = ms / args.steps
+    st = rb.read_stats(stats)
+    peak, peak_kind = load_peaks()
+    row_bytes = V * (2 if w.dtype == "bf16" else 4)
+    algo = live_rows * 2 * row_bytes + (T - live_rows) * row_bytes   # live rows: one read + one write
+    # reads grow with the live rows (the second sweep misses L2 for part of each), writes with all rows
+    traffic = TRAFFIC_OP_READ_PER_LIVE_BYTE * live_rows * row_bytes + TRAFFIC_OP_WRITE_PER_ROW_BYTE * T * row_bytes
+    ach = algo / (ms_per_step * 1e-3) / 1e9
+    line = {
+        "metric": "on-policy PG loss fwd+bwd tokens/sec at V=151936 bf16 (single pass)",
+        "value": tokens / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic", "ms_per_step_median": ms_median,
+        "config": {"workload": "onpolicy (slm mini-batch, mu = pi_theta)", "prompts": w.n_prompts,
+                   "generations_per_prompt": w.group_size, "padded_len": w.seq_len, "vocab": V,
+                   "logits_dtype": w.dtype, "unmasked_tokens_per_gpu": n_tokens, "live_rows_per_gpu": live_rows,
+                   "rows_per_gpu": T, "l2_policy": "inputs larger than L2",
+                   "parallelism": f"dp{world} (by prompt group, no data-path collective)"},
+        "clocks": clocks, "e2e": None, "gpu_launches": 4 * args.steps,
+        "roofline": {"bound": "hbm", "kernel": "onpolicy_rows_kernel", "achieved": ach, "peak": peak,
+                     "peak_kind": peak_kind, "unit": "GB/s", "frac": ach / peak, "frac_of_8TBs_nominal": ach / 8000.0,
+                     "achieved_at_median": algo / (ms_median * 1e-3) / 1e9,
+                     "algorithmic_bytes_per_launch": algo, "traffic": traffic, "traffic_source": TRAFFIC_OP_SOURCE},
+        "cpu_baseline": None, "stats": {"loss": st["loss"], "status": st["status"]},
+    }
+    return line
+
+
+# ------------------------------------------------------------------------------------------------
+# the other forms of the path, appended to the default line
+# ------------------------------------------------------------------------------------------------
+
+def run_extras(args, rk: Rank) -> dict:
+    """Short timed runs of the on-policy, fused-head (both variants) and long-sequence workloads, each
+    with the same timing protocol and its own clock record, condensed to one object per workload."""
+    import copy
+    import gc
+    out = {}
+    plan = [("roofline_onpolicy", run_onpolicy, {"workload": "onpolicy", "steps": 30}),
+            ("roofline_fused", run_fused, {"workload": "fused", "head": "recompute", "steps": 12}),
+            ("roofline_fused_stored", run_fused, {"workload": "fused", "head": "stored", "steps": 12}),
+            ("roofline_long", run_ours, {"workload": "long", "steps": 20})]
+    for key, fn, over in plan:
+        a = copy.copy(args)
+        for k, v in over.items():
+            setattr(a, k, v)
+        a.warmup, a.skip_e2e, a.seq_len, a.cpu_seconds = 3, True, 0, 4.0
+        gc.collect()
+        torch.cuda.empty_cache()
+        try:
+            ln = fn(a, rk)
+        except Exception as ex:      # a workload that cannot run here must not take the headline line down
+            out[key] = {"unavailable": f"{type(ex).__name__}: {str(ex).splitlines()[0][:200]}"}
+            continue
+        if ln is None:
+            continue
+        r = dict(ln["roofline"])
+        r.update({"workload": ln["config"]["workload"], "metric": ln["metric"], "value": ln["value"],
+                  "unit": ln["unit"], "steps": ln["steps"], "warmup": ln["warmup"], "ms_per_step": ln["ms_per_step"],
+                  "ms_per_step_median": ln.get("ms_per_step_median"), "clocks": ln["clocks"],
+                  "gpu_launches": ln["gpu_launches"], "cpu_baseline": ln.get("cpu_baseline")})
+        if "roofline_pass1" in ln:
+            r["pass1"] = ln["roofline_pass1"]
+            r["step"] = ln["roofline_step"]
+        out[key] = r
+    return out
 
 
 def main():
@@ -734,19 +846,37 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--skip-e2e", action="store_true", help="leave out the host-buffer leg (profiling)")
     ap.add_argument("--skip-cpu", action="store_true", help="leave out the CPU oracle timing (profiling)")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="default workload on one GPU: leave out the appended runs of the other workloads")
+    ap.add_argument("--cpu-seconds", type=float, default=10.0, help="size of the CPU oracle's timed sample")
     ap.add_argument("--seq-len", type=int, default=0,
                     help="shorter padded length (smaller device footprint, e.g. for profiling)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
-    else:
-        args.warmup = max(args.warmup, 3)
+        return
+    what, arg = launch_command(args.gpus, os.environ, sys.argv[1:],
+                               torch.cuda.device_count() if torch.cuda.is_available() else 0, free_port())
+    if what == "error":
+        raise SystemExit("bench.py: " + arg)
+    if what == "exec":
+        sys.stdout.flush()
+        os.execv(arg[0], arg)
+    args.warmup = max(args.warmup, 3)
+    rk = Rank()
+    try:
         if args.workload == "fused":
-            run_fused(args)
+            line = run_fused(args, rk)
         elif args.workload == "onpolicy":
-            run_onpolicy(args)
+            line = run_onpolicy(args, rk)
         else:
-            run_ours(args)
+            line = run_ours(args, rk)
+        if args.workload == "slm" and rk.world == 1 and not args.no_extras and not args.seq_len:
+            line.update(run_extras(args, rk))
+        if rk.rank == 0:
+            print(json.dumps(line), flush=True)
+    finally:
+        rk.close()
 
 
 if __name__ == "__main__":

@@ -227,6 +227,23 @@ def head_logits(hidden_bits: np.ndarray, w_bits: np.ndarray, rows=None) -> np.nd
     return out
 
 
+def decode_bf16(bits: np.ndarray) -> np.ndarray:
+    """bf16 bit patterns (uint16) -> the float64 values they stand for (exact)."""
+    bits = _c(bits, np.uint16)
+    return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def head_logits_dgemm(hidden_bits: np.ndarray, w_f64: np.ndarray, rows=None) -> np.ndarray:
+    """z[rows] = h[rows] @ W in float64 with the library's matrix product as the step.
+
+    Same definition as head_logits (the fused-head form's z = h W); the sum over the hidden
+    dimension is taken by float64 GEMM instead of the plain loops, which is what makes all
+    16 384 rows of the full-size configuration affordable (3.8e12 multiply-adds).  `w_f64` is
+    decode_bf16(w_bits), decoded once by the caller.  The two differ only in summation order."""
+    h = decode_bf16(hidden_bits if rows is None else _c(hidden_bits, np.uint16)[_c(rows, np.int64)])
+    return h @ w_f64
+
+
 def token_logp_f64(z: np.ndarray, targets_of_list):
     z = _c(z, np.float64)
     n, V = z.shape

@@ -46,31 +46,76 @@ struct FloatSum {
     __device__ __forceinline__ double value() const { return (double)s + (double)c; }
 };
 
+// A thread's state is (m, sh, S, T): the largest logit seen, the shift sh = ceil(fl(m k)) with
+// k = fl(log2 e) that its exponentials were taken against (an integer, so that moving to a new shift
+// multiplies by an exact power of two) plus a 16-bit fraction `off` that differs from thread to
+// thread, S = sum_v e_v with e_v = 2^(x_v), x_v = z_v k - sh, and
+// T = sum_v x_v e_v.  Three things keep the log-sum-exp free of any bias beyond a few 1e-9, which a
+// generation-level weight multiplies by the generation's length:
+//  * the shift is USED as it stands, in the exponentials and again when threads are combined, and
+//    turned back into natural-log units as sh / k, so no rounding of m k enters;
+//  * k differs from log2(e) by rho = 1.3e-8 (relative), so the wanted term is 2^(x (1 + rho)) =
+//    e_v (1 + rho ln2 x_v): the first-order correction rho ln2 T is added to S at the end;
+//  * the hardware exponential's relative error on negative arguments, averaged over the fraction of
+//    the argument, is kEx2Bias (measured over all 2^23 fractions on sm_100a: -5.0e-8, the same to 3 %
+//    for every integer part; errors lie in [-1.44e-7, +0.63e-7]); a sum of many terms carries that
+//    mean, and is divided by 1 + kEx2Bias.  bf16 logits take few distinct values and k is fixed, so
+//    with a common integer shift the fraction of x_v would depend on z_v alone and the sum would carry
+//    the errors of those few fractions (a bias of 1e-8 either way) instead of the mean; the per-thread
+//    fraction of the shift spreads every logit value over 128 different fractions.
+//  * the thread's largest logit, which may carry nearly all of the row's probability, gets no such
+//    statistical treatment: its hardware exponential is taken out of S and T again at the end of the
+//    sweep and replaced by the exact value in double.
+constexpr float kEx2Bias = -5.0e-8f;
+constexpr double kLog2eF = (double)kLog2e;                       // the float constant, exactly
+constexpr double kOnePlusRho = kLog2eD / kLog2eF;
+constexpr double kRhoLn2 = (kLog2eD - kLog2eF) / kLog2eF * kLn2D;  // rho ln 2
+
 template <int U>
-__device__ __forceinline__ void bf16_batch(const uint4 (&q)[U], float& m, FloatSum& S) {
+__device__ __forceinline__ void bf16_batch(const uint4 (&q)[U], float off, float& m, float& sh, FloatSum& S,
+                                           float& T) {
     uint32_t mx = bf16x2_max(bf16x2_max(q[0].x, q[0].y), bf16x2_max(q[0].z, q[0].w));
 #pragma unroll
     for (int j = 1; j < U; ++j)
         mx = bf16x2_max(mx, bf16x2_max(bf16x2_max(q[j].x, q[j].y), bf16x2_max(q[j].z, q[j].w)));
     const float bm = fmaxf(bf16_lo(mx), bf16_hi(mx));
-    if (bm > m) {  // rare after the first few batches
-        S.scale(ex2_approx((m - bm) * kLog2e));
-        m = bm;
-    }
     // logits may be -inf or the lowest finite value (a masked part of the vocabulary): while the thread
-    // has seen nothing else its maximum is that too, and the shift -m log2(e) must neither turn
-    // (-inf) - (-inf) into a NaN nor overflow to +inf
-    const float nm = (m < -1.0e38f) ? 0.f : -m * kLog2e;
-    float s0 = 0.f, s1 = 0.f;
+    // has seen nothing else it keeps the shift 0, so that the shift neither turns (-inf) - (-inf) into
+    // a NaN nor overflows to +inf
+    if (bm > m) {  // rare after the first few batches
+        m = bm;
+        if (bm > -1.0e38f) {
+            const float nsh = ceilf(bm * kLog2e) + off;
+            const float f = ex2_approx(sh - nsh);  // exact: an integer power of two (and S = T = 0 for an empty thread)
+            T = f * fmaf(sh - nsh, S.s, T);        // every x moves by sh - nsh
+            S.scale(f);
+            sh = nsh;
+        }
+    }
+    // a pair of logits at a time in the packed two-float forms (one instruction for two multiply-adds
+    // or two additions, each rounded like its scalar form).  Masked entries (-inf, or the lowest finite
+    // value) are raised to -1e30 first: their exponential is still exactly 0, and 0 * x stays 0 in T.
+    const uint64_t k2 = f32x2(kLog2e, kLog2e), nsh2 = f32x2(-sh, -sh);
+    constexpr uint32_t kFloor2 = 0xf14af14au;  // bf16 pair (-1.0e30, -1.0e30)
+    uint64_t s2 = f32x2(0.f, 0.f), t2 = f32x2(0.f, 0.f);
 #pragma unroll
     for (int j = 0; j < U; ++j) {
         const uint32_t w[4] = {q[j].x, q[j].y, q[j].z, q[j].w};
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            s0 += ex2_approx(fmaf(bf16_lo(w[k]), kLog2e, nm));
-            s1 += ex2_approx(fmaf(bf16_hi(w[k]), kLog2e, nm));
+            const uint32_t z2 = bf16x2_max(w[k], kFloor2);
+            const uint64_t x2 = f32x2_fma(f32x2(bf16_lo(z2), bf16_hi(z2)), k2, nsh2);
+            float x0, x1;
+            f32x2_split(x2, x0, x1);
+            const uint64_t e2 = f32x2(ex2_approx(x0), ex2_approx(x1));
+            s2 = f32x2_add(s2, e2);
+            t2 = f32x2_fma(x2, e2, t2);
         }
     }
+    float s0, s1, t0, t1;
+    f32x2_split(s2, s0, s1);
+    f32x2_split(t2, t0, t1);
+    T += t0 + t1;
     const float b = s0 + s1;
     if (b > S.s) {  // keep the larger operand first, as Fast2Sum wants (early batches only)
         const float old = S.s;
@@ -83,15 +128,20 @@ __device__ __forceinline__ void bf16_batch(const uint4 (&q)[U], float& m, FloatS
 
 // `out`, when not null, receives a copy of the row (same layout): used when the logits are read from
 // host memory and the second pass wants them on the device.
-__device__ __forceinline__ void row_sweep_bf16(const uint16_t* row, int vocab, float& m_out,
+// Returns the thread's maximum, its shift (log2 units) and its share of sum_v exp(z_v - sh / k), all
+// corrections applied; a thread that saw nothing real returns 0 and the shift 0.
+__device__ __forceinline__ void row_sweep_bf16(const uint16_t* row, int vocab, float& m_out, float& sh_out,
                                                double& s_out, uint16_t* out) {
     constexpr int U = RAPID_P1_U;
     const int tid = threadIdx.x;
     const int nvec = vocab >> 3;
     const uint4* rv = reinterpret_cast<const uint4*>(row);
     uint4* ov = reinterpret_cast<uint4*>(out);
-    float m = -INFINITY;
+    float m = -INFINITY, sh = 0.f, T = 0.f;
     FloatSum S{0.f, 0.f};
+    // this thread's fraction of the shift (see above): 16 bits, scattered, so that the fractions neither
+    // line up with a table of the hardware exponential nor cost the shift its exactness
+    const float off = (float)(((unsigned)tid * 40503u) & 0xffffu) * (1.f / 65536.f);
     int v = tid;
     for (; v + (U - 1) * kThreads < nvec; v += U * kThreads) {
         uint4 q[U];
@@ -101,29 +151,48 @@ __device__ __forceinline__ void row_sweep_bf16(const uint16_t* row, int vocab, f
 #pragma unroll
             for (int j = 0; j < U; ++j) ov[v + j * kThreads] = q[j];
         }
-        bf16_batch<U>(q, m, S);
+        bf16_batch<U>(q, off, m, sh, S, T);
     }
     for (; v < nvec; v += kThreads) {
         uint4 q[1];
         q[0] = ld_stream(rv + v);
         if (out) ov[v] = q[0];
-        bf16_batch<1>(q, m, S);
+        bf16_batch<1>(q, off, m, sh, S, T);
     }
     // ragged tail (vocab not a multiple of 8): one element per thread
-    double tail = 0.0;
+    double tail = 0.0, tail_t = 0.0;
     const int e = (nvec << 3) + tid;
     if (e < vocab) {
         const uint16_t zb = row[e];
         if (out) out[e] = zb;
         const float z = __uint_as_float(((uint32_t)zb) << 16);
         if (z > m) {
-            S.scale(ex2_approx((m - z) * kLog2e));
             m = z;
+            if (z > -1.0e38f) {
+                const float nsh = ceilf(z * kLog2e) + off;
+                const float f = ex2_approx(sh - nsh);
+                T = f * fmaf(sh - nsh, S.s, T);
+                S.scale(f);
+                sh = nsh;
+            }
         }
-        if (z != -INFINITY) tail = (double)ex2_approx((z - m) * kLog2e);
+        if (z > -1.0e38f) {
+            const float x = fmaf(z, kLog2e, -sh);
+            tail = (double)ex2_approx(x);
+            tail_t = (double)fmaxf(x, -200.f) * tail;
+        }
     }
     m_out = m;
-    s_out = S.value() + tail;
+    sh_out = sh;
+    double s = S.value() + tail, t = (double)T + tail_t, top = 0.0;
+    if (m > -1.0e38f) {  // the largest logit: out with what the hardware gave for it, in with the exact term
+        const float xm = fmaf(m, kLog2e, -sh);
+        const float em = ex2_approx(xm);
+        s -= (double)em;
+        t -= (double)xm * (double)em;
+        top = exp2(((double)m * kLog2eF - (double)sh) * kOnePlusRho);
+    }
+    s_out = (s + kRhoLn2 * t) / (1.0 + (double)kEx2Bias) + top;
 }
 
 // ---- fp32 ------------------------------------------------------------------------------------
@@ -192,6 +261,7 @@ row_stats_kernel(const void* __restrict__ logits, void* __restrict__ copy_out, i
                  int64_t n_rows, const int32_t* __restrict__ targets,
                  const uint8_t* __restrict__ mask, Workspace ws) {
     __shared__ float sh_m[kWarps];
+    __shared__ float sh_sh[kWarps];
     __shared__ double sh_s[kWarps];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
@@ -210,31 +280,39 @@ row_stats_kernel(const void* __restrict__ logits, void* __restrict__ copy_out, i
         }
 
         float M;
-        double S;  // sum_v exp(z_v - M) for this thread's share, then the row
+        double S;      // the row's sum of exponentials against `shift`
+        double shift;  // M for float logits; the float shift actually used, in natural-log units, for bf16
         double zy;
         if (DT == RAPID_BF16) {
             const uint16_t* row = static_cast<const uint16_t*>(logits) + i * ld;
-            float m;
+            float m, sh;
             double s;
             uint16_t* orow = copy_out ? static_cast<uint16_t*>(copy_out) + i * ld : nullptr;
-            row_sweep_bf16(row, vocab, m, s, orow);
+            row_sweep_bf16(row, vocab, m, sh, s, orow);
+            // threads are brought to a common shift in double, with the shifts exactly as they were used;
+            // a thread (or a whole warp, for a tiny vocabulary) that saw nothing has s = 0
             const float wm = warp_max(m);
-            // a thread (or a whole warp, for a tiny vocabulary) that saw nothing has m = -inf, s = 0
-            if (m != wm) s *= (double)ex2_approx((m - wm) * kLog2e);
+            const float wsh = warp_max(s > 0.0 ? sh : -INFINITY);
+            if (s > 0.0 && sh != wsh) s *= exp2(((double)sh - (double)wsh) * kOnePlusRho);
             s = warp_sum(s);
             if (lane == 0) {
                 sh_m[warp] = wm;
+                sh_sh[warp] = wsh;
                 sh_s[warp] = s;
             }
             __syncthreads();
             if (tid == 0) {
-                float mm = sh_m[0];
-                for (int w = 1; w < kWarps; ++w) mm = fmaxf(mm, sh_m[w]);
+                float mm = sh_m[0], msh = sh_sh[0];
+                for (int w = 1; w < kWarps; ++w) {
+                    mm = fmaxf(mm, sh_m[w]);
+                    msh = fmaxf(msh, sh_sh[w]);
+                }
                 double tot = 0.0;
                 for (int w = 0; w < kWarps; ++w)
-                    tot += sh_s[w] * (double)ex2_approx((sh_m[w] - mm) * kLog2e);
+                    if (sh_s[w] > 0.0) tot += sh_s[w] * exp2(((double)sh_sh[w] - (double)msh) * kOnePlusRho);
                 M = mm;
                 S = tot;
+                shift = (double)msh / kLog2eF;  // lse = shift + log(S)
                 zy = (double)__uint_as_float(((uint32_t)row[y]) << 16);  // (one more 2-byte read of the row)
             }
         } else {
@@ -260,11 +338,12 @@ row_stats_kernel(const void* __restrict__ logits, void* __restrict__ copy_out, i
                     if (sh_s[w] > 0.0) tot += sh_s[w] * exp((double)sh_m[w] - (double)mm);
                 M = mm;
                 S = tot;
+                shift = (double)mm;
                 zy = (double)row[y];
             }
         }
         if (tid == 0) {
-            const double lse = (double)M + log(S);
+            const double lse = shift + log(S);
             ws.lse[r] = lse;
             ws.token_logp[r] = zy - lse;
             ws.row_max[r] = M;

@@ -19,7 +19,7 @@ pytestmark = pytest.mark.gpu
 import oracle  # noqa: E402
 from paper_2510_03515_b200 import binding as rb  # noqa: E402
 from paper_2510_03515_b200 import synth  # noqa: E402
-from parity_util import DLOGITS_ATOL, LOGP_ATOL, LOSS_RTOL, adv_atol  # noqa: E402
+from parity_util import DLOGITS_ATOL, LOGP_ATOL, LOSS_RTOL, adv_atol, report_observed  # noqa: E402
 
 
 def _oracle_steps_2_to_5(w, tok, lp, row_ok, behav, eta=2.0, flags=0):
@@ -66,55 +66,93 @@ def _property_checks(dz, live_row, dt, block=4096):
         assert blk.sum(1).abs().max().item() <= tol
 
 
-@pytest.mark.parametrize("name,sigma", [("slm", None), ("stale", 0.5)])
-def test_resident_batch_full_size(name, sigma):
-    w = synth.CONFIGS[name]
-    if sigma is not None:
-        w = w.scaled(behav_sigma=sigma)
+def _resident_batch_full_size(w, cases):
+    """`cases`: list of (label, sigma, shift) -- behaviour log-probs = the oracle's current ones +
+    N(0, sigma) + shift[n] per token of generation n.  Step 1 of the oracle (and the logits) do not
+    depend on the behaviour policy, so they are computed once and shared by all cases."""
     dt = synth.torch_dtype(w)
     dev = torch.device("cuda")
-    tok = synth.make_tokens(w)
+    tok = synth.make_tokens(w.scaled(behav_sigma=1.0))           # unit noise, scaled per case below
     T, V, N = w.n_rows, w.vocab, w.n_seq
     logits = synth.logits_for_sequences(w, tok["targets"], 0, N, device=dev)
     host = logits.cpu()
     bits = synth.bits_numpy(host)
     pre = oracle.token_logp(bits, V, tok["targets"].numpy(), tok["mask"].numpy())
-    behav = (torch.from_numpy(pre["token_logp"]) + tok["behav_noise"].double()).float()
-    o = _oracle_steps_2_to_5(w, tok, pre["token_logp"], pre["row_ok"], behav.numpy())
-
     targets, mask = tok["targets"].to(dev), tok["mask"].to(dev)
     desc = rb.make_desc(N, w.seq_len, V, w.n_prompts, dt, logits.stride(0), 2.0, 0)
     ws = rb.alloc_workspace(desc, dev)
     dz = torch.empty_like(logits)
-    loss = torch.zeros(1, device=dev)
-    tl = torch.empty(T, device=dev)
-    adv = torch.empty(N, device=dev)
-    stats = rb.alloc_stats(dev)
-    rb.rapid_pg_stats_chunk(desc, logits, 0, T, targets, mask, ws)
-    rb.rapid_pg_finalize(desc, behav.to(dev), tok["rewards"].to(dev), tok["group_offsets"].to(dev), loss,
-                         tl, adv, stats, ws)
-    rb.rapid_pg_dlogits_chunk(desc, logits, dz, 0, T, targets, stats, ws)
-    torch.cuda.synchronize()
-
-    np.testing.assert_allclose(tl.cpu().numpy(), pre["token_logp"], rtol=0, atol=LOGP_ATOL[dt])
-    _check_scalars(o, loss.item(), adv.cpu().numpy(), rb.read_stats(stats), dt, w.seq_len)
-    assert torch.equal(logits.cpu(), host), "logits modified"
-
     rows = _sample_rows(w, tok, 3000, seed=w.seed)
-    worst = 0.0
-    for i in range(0, len(rows), 256):
-        sel = rows[i:i + 256]
-        ref = oracle.dlogits_rows(bits, V, w.seq_len, tok["targets"].numpy(), pre["row_ok"], pre["lse"],
-                                  o["coef"], sel)
-        got = dz[torch.from_numpy(sel).to(dev)].float().cpu().numpy().astype(np.float64)
-        worst = max(worst, float(np.abs(got - ref).max()))
-    assert worst <= DLOGITS_ATOL[dt], f"dlogits max abs err {worst}"
+    outs = {}
+    for label, sigma, shift in cases:
+        noise = tok["behav_noise"].double() * sigma
+        if shift is not None:
+            noise = noise + torch.from_numpy(np.repeat(shift, w.seq_len))
+        behav = (torch.from_numpy(pre["token_logp"]) + noise).float()
+        o = _oracle_steps_2_to_5(w, tok, pre["token_logp"], pre["row_ok"], behav.numpy())
 
-    live = torch.from_numpy(pre["row_ok"].astype(bool) & (np.repeat(o["coef"], w.seq_len) != 0.0)).to(dev)
-    _property_checks(dz, live, dt)
-    if name == "stale":
+        loss = torch.zeros(1, device=dev)
+        tl = torch.empty(T, device=dev)
+        adv = torch.empty(N, device=dev)
+        stats = rb.alloc_stats(dev)
+        dz.fill_(float("nan"))
+        rb.rapid_pg_stats_chunk(desc, logits, 0, T, targets, mask, ws)
+        rb.rapid_pg_finalize(desc, behav.to(dev), tok["rewards"].to(dev), tok["group_offsets"].to(dev), loss,
+                             tl, adv, stats, ws)
+        rb.rapid_pg_dlogits_chunk(desc, logits, dz, 0, T, targets, stats, ws)
+        torch.cuda.synchronize()
+
+        np.testing.assert_allclose(tl.cpu().numpy(), pre["token_logp"], rtol=0, atol=LOGP_ATOL[dt])
+        st = rb.read_stats(stats)
+        _check_scalars(o, loss.item(), adv.cpu().numpy(), st, dt, w.seq_len)
+
+        worst = 0.0
+        for i in range(0, len(rows), 256):
+            sel = rows[i:i + 256]
+            ref = oracle.dlogits_rows(bits, V, w.seq_len, tok["targets"].numpy(), pre["row_ok"], pre["lse"],
+                                      o["coef"], sel)
+            got = dz[torch.from_numpy(sel).to(dev)].float().cpu().numpy().astype(np.float64)
+            worst = max(worst, float(np.abs(got - ref).max()))
+        assert worst <= DLOGITS_ATOL[dt], f"{label}: dlogits max abs err {worst}"
+
+        live = torch.from_numpy(pre["row_ok"].astype(bool) & (np.repeat(o["coef"], w.seq_len) != 0.0)).to(dev)
+        _property_checks(dz, live, dt)
+        scale = max(abs(o["loss"]), 1e-3 * float(np.abs(o["coef"] * o["seq_logp"]).sum()), 1e-30)
+        report_observed(f"{w.name} full size, {label}", loss=abs(loss.item() - o["loss"]) / scale / LOSS_RTOL[dt],
+                        token_logp=np.abs(tl.cpu().numpy() - pre["token_logp"]).max() / LOGP_ATOL[dt],
+                        adv=np.abs(adv.cpu().numpy() - o["adv64"]).max() / adv_atol(dt, w.seq_len),
+                        dlogits=worst / DLOGITS_ATOL[dt])
+        outs[label] = (o, st)
+    assert torch.equal(logits.cpu(), host), "logits modified"
+    return outs
+
+
+def test_slm_batch_full_size():
+    w = synth.CONFIGS["slm"]
+    _resident_batch_full_size(w, [("sigma 0.2", w.behav_sigma, None)])
+
+
+def test_staleness_sweep_full_size():
+    """128 x 512 tokens at every staleness level of the sweep, sigma in {0, 0.1, 0.5, 1, 2}: from
+    weights that are all one to log-weights with a standard deviation of 2 sqrt(512) = 45, where
+    nearly every weight is either clipped at eta or vanishes.  A sixth case shifts three
+    generations' behaviour log-probs by -2 per token, so that their log-weight passes 709 and the
+    exponential overflows to +inf in double precision, which the clip turns into eta."""
+    w = synth.CONFIGS["stale"]
+    shift = np.zeros(w.n_seq)
+    shift[[20, 21, 77]] = -2.0                                   # members of groups 2 and 9
+    cases = [(f"sigma {s:g}", s, None) for s in synth.STALE_SIGMAS] + [("sigma 2 + overflow", 2.0, shift)]
+    outs = _resident_batch_full_size(w, cases)
+    for label, (o, st) in outs.items():
         assert np.all(o["adv64"][:w.group_size] == 0.0)          # the all-zero-reward group
-        assert o["stats"]["n_clipped"] > 0
+        assert np.all(np.isfinite(o["coef"])) and np.isfinite(o["loss"])
+    o0, st0 = outs["sigma 0"]
+    assert st0["n_clipped"] == 0 and abs(st0["mean_log_cw"]) < 1e-3 and np.all(np.abs(o0["weight"] - 1.0) < 1e-3)
+    o2, st2 = outs["sigma 2"]
+    assert o2["weight"].max() > 3.4e38, "some weight should lie beyond the float32 range at sigma = 2"
+    assert st2["n_clipped"] >= w.n_seq // 4
+    oo, sto = outs["sigma 2 + overflow"]
+    assert np.isinf(oo["weight"][[20, 21, 77]]).all() and sto["n_clipped"] == oo["stats"]["n_clipped"]
 
 
 def test_long_config_full_size_chunked():
@@ -171,3 +209,8 @@ def test_long_config_full_size_chunked():
         _property_checks(buf, torch.from_numpy(live_all[r0:r0 + nr]).to(dev), dt)
     assert worst <= DLOGITS_ATOL[dt], f"dlogits max abs err {worst}"
     assert rb.read_stats(stats)["status"] == 0
+    scale = max(abs(o["loss"]), 1e-3 * float(np.abs(o["coef"] * o["seq_logp"]).sum()), 1e-30)
+    report_observed("long full size (chunked)", loss=abs(loss.item() - o["loss"]) / scale / LOSS_RTOL[dt],
+                    token_logp=np.abs(tl.cpu().numpy() - lp).max() / LOGP_ATOL[dt],
+                    adv=np.abs(adv.cpu().numpy() - o["adv64"]).max() / adv_atol(dt, L),
+                    dlogits=worst / DLOGITS_ATOL[dt])

@@ -11,7 +11,7 @@ pytestmark = pytest.mark.gpu
 import oracle  # noqa: E402
 from paper_2510_03515_b200 import binding as rb  # noqa: E402
 from paper_2510_03515_b200 import synth  # noqa: E402
-from parity_util import compare, run_both  # noqa: E402
+from parity_util import compare, report_observed, run_both  # noqa: E402
 
 
 def _dt(w):
@@ -25,6 +25,8 @@ def test_config_tiny_full_size():
     o, g = run_both(b, w.n_seq, w.seq_len)
     r = compare(o, g, _dt(w), w.seq_len)
     assert np.abs(g["dlogits"].sum(1)).max() < 1e-6
+    report_observed("tiny (every element)", loss=r["loss_vs_bound"], token_logp=r["logp_vs_bound"],
+                    adv=r["adv_vs_bound"], dlogits=r["dlogits_vs_bound"])
 
 
 @pytest.mark.parametrize("in_place", [False, True])
@@ -34,8 +36,10 @@ def test_config_slm_scaled(in_place):
     w = synth.CONFIGS["slm"].scaled(n_prompts=2, group_size=4, seq_len=40, len_lo=10)
     b = synth.make_batch(w)
     o, g = run_both(b, w.n_seq, w.seq_len, in_place=in_place)
-    compare(o, g, _dt(w), w.seq_len)
+    r = compare(o, g, _dt(w), w.seq_len)
     assert (b["mask"] == 0).any()
+    report_observed(f"slm scaled (every element, in_place={in_place})", loss=r["loss_vs_bound"],
+                    token_logp=r["logp_vs_bound"], adv=r["adv_vs_bound"], dlogits=r["dlogits_vs_bound"])
 
 
 @pytest.mark.parametrize("sigma", synth.STALE_SIGMAS)

@@ -608,6 +608,29 @@ def test_head_functions_against_matmul_and_fd(oracle):
     np.testing.assert_allclose(dW, fd_W, atol=1e-8)
 
 
+def test_head_logits_dgemm_is_the_same_product(oracle):
+    """The library-matmul form of z = h W against (i) a case whose every product and partial sum is
+    an exact small integer, so any summation order gives the same bits, and (ii) the plain loops on
+    random bf16 inputs, where the two may differ by summation order only."""
+    h_int = np.array([[1, -2, 3], [0, 4, -1]], np.float64)
+    W_int = np.array([[2, 0, -1, 5], [1, 1, 3, -2], [-4, 2, 0, 1]], np.float64)
+    z = oracle.head_logits_dgemm(bf16_bits(h_int), oracle.decode_bf16(bf16_bits(W_int)))
+    np.testing.assert_array_equal(z, [[-12, 4, -7, 12], [8, 2, 12, -9]])
+    np.testing.assert_array_equal(oracle.head_logits(bf16_bits(h_int), bf16_bits(W_int)), z)
+
+    rng = np.random.default_rng(43)
+    T, D, V = 37, 96, 301
+    h_bits = bf16_bits(rng.normal(0, 1, (T, D)))
+    w_bits = bf16_bits(rng.normal(0, 0.02, (D, V)))
+    np.testing.assert_array_equal(oracle.decode_bf16(w_bits), bf16_to_f64(w_bits))
+    plain = oracle.head_logits(h_bits, w_bits)
+    fast = oracle.head_logits_dgemm(h_bits, oracle.decode_bf16(w_bits))
+    mag = np.abs(bf16_to_f64(h_bits)) @ np.abs(bf16_to_f64(w_bits))
+    assert (np.abs(fast - plain) <= 4 * D * 2.0 ** -53 * mag).all()
+    rows = np.array([30, 2, 2, 17], np.int64)
+    np.testing.assert_array_equal(oracle.head_logits_dgemm(h_bits, oracle.decode_bf16(w_bits), rows), fast[rows])
+
+
 # --------------------------------------------------------------------------------------------
 # structural properties of the whole path (none of them is the oracle's own formula restated)
 # --------------------------------------------------------------------------------------------
