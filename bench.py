@@ -822,7 +822,7 @@ def run_extras(args, rk: Rank) -> dict:
             continue
         r = dict(ln["roofline"])
         r.update({"workload": ln["config"]["workload"], "metric": ln["metric"], "value": ln["value"],
-                  "unit": ln["unit"], "steps": ln["steps"], "warmup": ln["warmup"], "ms_per_step": ln["ms_per_step"],
+                  "value_unit": ln["unit"], "steps": ln["steps"], "warmup": ln["warmup"], "ms_per_step": ln["ms_per_step"],
                   "ms_per_step_median": ln.get("ms_per_step_median"), "clocks": ln["clocks"],
                   "gpu_launches": ln["gpu_launches"], "cpu_baseline": ln.get("cpu_baseline")})
         if "roofline_pass1" in ln:

@@ -28,7 +28,9 @@
  * Conventions, unless a parameter says otherwise:
  *   - `desc`, `bytes` and other plain scalars are HOST memory; every array pointer is a DEVICE
  *     pointer owned by the caller and valid on the current device.  The library allocates
- *     nothing, keeps no state between calls and frees nothing.
+ *     nothing, frees nothing and keeps no state between calls: everything a call needs beyond its
+ *     arguments lives in the caller's workspace.  (One exception, stated at its declaration:
+ *     rapid_pg_loss_fwd_bwd_noalloc works in a fixed device array that all its calls share.)
  *   - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = the default stream)
  *     and the call returns without synchronising.  Outputs are valid once the stream reaches
  *     the end of the enqueued work.
@@ -37,7 +39,9 @@
  *     [0, vocab) makes its row count as masked and is counted in rapid_stats_t.n_bad_token; an
  *     invalid group_offsets array sets rapid_stats_t.status, zeroes every coefficient (so
  *     dlogits is all zero) and makes loss NaN.
- *   - Logits must be finite.  +-inf or NaN logits give unspecified (but memory-safe) results.
+ *   - Logits must not be +inf or NaN (results unspecified, but memory-safe).  -inf, or the
+ *     dtype's lowest finite value, marks a masked part of the vocabulary and is accepted under the
+ *     condition stated at rapid_pg_loss_fwd_bwd.
  *   - Only sm_100 devices are supported: other devices get RAPID_ERR_UNSUPPORTED.
  */
 #ifndef RAPID_PG_H
@@ -114,6 +118,19 @@ typedef struct rapid_stats {
     double mean_abs_log_cw; /* (1/N) sum_n |log c_n|                                              */
     double loss;            /* the loss in double                                                 */
 } rapid_stats_t;
+
+/*
+ * Self-test of the time-out path (the paper has no counterpart: this is a property of the
+ * implementation).  The pipelined kernels wait on shared-memory barriers for their bulk copies;
+ * every such wait is bounded and, when its limit passes, raises RAPID_ERR_TIMEOUT in the statistics
+ * block instead of spinning or trapping.  This call runs that very wait routine in a one-warp kernel
+ * on a barrier that nothing arrives at, with a limit of `limit_ns` nanoseconds (1 .. 1e9; more
+ * returns RAPID_ERR_UNSUPPORTED, 0 or a NULL `stats` RAPID_ERR_INVALID_ARG).  On completion
+ * stats->status == RAPID_ERR_TIMEOUT and stats->n_tokens holds the nanoseconds the wait lasted;
+ * the other fields are zero.  `stats` is a DEVICE pointer.  The kernel ends normally and the context
+ * stays usable.
+ */
+rapid_status_t rapid_selftest_bounded_wait(uint64_t limit_ns, rapid_stats_t* stats, void* stream);
 
 /* Human-readable name of a status code (static storage, never NULL). */
 const char* rapid_status_string(rapid_status_t status);
@@ -201,9 +218,11 @@ rapid_status_t rapid_pg_loss_fwd_bwd(const rapid_desc_t* desc, const void* logit
  *     (about 21 bytes per row of the token grid, i.e. up to roughly 199 000 rows).  Anything
  *     larger returns RAPID_ERR_UNSUPPORTED and enqueues nothing; use the workspace form instead.
  *   - The call allocates and frees nothing, on the device or through any library.
- *   - First call on each device: the library looks up the device address of its array (a
- *     cudaGetSymbolAddress call, made with the caller's current device) and remembers it.  Make
- *     this first call, on every device you will use, before beginning any stream capture.
+ *   - Every call looks up the device address of the array for the caller's current device (a
+ *     cudaGetSymbolAddress call) and remembers nothing, so the call stays valid after a
+ *     cudaDeviceReset and under whichever context is current.  The FIRST call on a device is the
+ *     one that makes the runtime set the array up there: make it, on every device you will use,
+ *     before beginning any stream capture.
  *   - All calls on a device share the one array, and it keeps whatever the previous call left in
  *     it.  Nothing in it needs clearing between calls (each call rewrites what it reads), but two
  *     calls whose GPU work can overlap -- different streams, or different host threads without

@@ -41,7 +41,7 @@ EXPORTS = (
     "rapid_status_string", "rapid_version", "rapid_workspace_bytes", "rapid_group_advantage",
     "rapid_pg_loss_fwd_bwd", "rapid_pg_stats_chunk", "rapid_pg_finalize", "rapid_pg_dlogits_chunk",
     "rapid_pg_loss_fwd_bwd_noalloc", "rapid_fused_head_workspace_bytes", "rapid_pg_loss_fused_head",
-    "rapid_pg_loss_onpolicy_fwd_bwd", "rapid_pg_loss_fwd_bwd_hostlogits",
+    "rapid_pg_loss_onpolicy_fwd_bwd", "rapid_pg_loss_fwd_bwd_hostlogits", "rapid_selftest_bounded_wait",
 )
 
 
@@ -99,6 +99,8 @@ def lib():
         L.rapid_fused_head_workspace_bytes.argtypes = [dp, C.c_int32, C.POINTER(C.c_size_t)]
         L.rapid_pg_loss_fused_head.restype = C.c_int
         L.rapid_pg_loss_fused_head.argtypes = [dp, C.c_int32] + [vp] * 14 + [sz, vp]
+        L.rapid_selftest_bounded_wait.restype = C.c_int
+        L.rapid_selftest_bounded_wait.argtypes = [C.c_uint64, vp, vp]
         L.rapid_pg_stats_chunk.restype = C.c_int
         L.rapid_pg_stats_chunk.argtypes = [dp, vp, i64, i64, vp, vp, vp, sz, vp]
         L.rapid_pg_finalize.restype = C.c_int
@@ -253,6 +255,10 @@ def rapid_pg_loss_onpolicy_fwd_bwd(desc: RapidDesc, logits: torch.Tensor, target
         C.byref(desc), _ptr(logits), _ptr(targets), _ptr(mask), _ptr(rewards), _ptr(group_offsets),
         _ptr(dlogits), _ptr(loss), _ptr(token_logp), _ptr(adv), _ptr(stats), _ptr(workspace),
         workspace.numel(), _stream()), "rapid_pg_loss_onpolicy_fwd_bwd")
+
+
+def rapid_selftest_bounded_wait(limit_ns: int, stats: torch.Tensor) -> None:
+    _check(lib().rapid_selftest_bounded_wait(int(limit_ns), _ptr(stats), _stream()), "rapid_selftest_bounded_wait")
 
 
 def rapid_fused_head_workspace_bytes(desc: RapidDesc, hidden_dim: int) -> int:

@@ -1,5 +1,6 @@
 // The C ABI of librapid_pg: host-side argument checks, workspace carving and kernel launches.
-// Nothing here allocates, synchronises or keeps state; see include/rapid_pg.h for the contract.
+// Nothing here allocates, synchronises or keeps state (the one call that works in a library-owned
+// array is in noalloc.cu); see include/rapid_pg.h for the contract.
 #include <math.h>
 
 #include "rapid_common.cuh"

@@ -18,9 +18,8 @@
 //                     bursts of kChunk bytes.  A chunk is fully read before any of it is
 //                     overwritten, so dlogits may be the logits buffer itself.
 //
-// bf16: g_n is folded into the exponent, dz = sign(g) 2^(z log2(e) - lse log2(e) + log2|g|), so the
-// inner loop is one fused multiply-add and one MUFU exponential per element.
-// fp32: p = exp((z - M) - (lse - M)) with the accurate exponential, then times g.
+// The arithmetic of one vector of a row is in dz_rows.cuh (shared with the on-policy kernel).
+#include "dz_rows.cuh"
 #include "rapid_common.cuh"
 #include "tma_pipe.cuh"
 
@@ -52,87 +51,6 @@ static_assert(kStages >= 3, "need a stage to load, one to work on and one to sto
 
 constexpr int kZeroThreads = 128;
 constexpr int kZeroBuf = 16384;
-
-__device__ __forceinline__ uint16_t float_to_bf16_bits(float x) {
-    return (uint16_t)(pack_bf16x2(x, 0.f) & 0xffffu);
-}
-
-struct RowConstBf16 {
-    float c;         // -lse log2(e) + log2|g|
-    float g;         // coefficient
-    uint32_t sign2;  // sign of g on both halves of a packed pair
-    int y;
-};
-struct RowConstF32 {
-    float M, a, g;  // row max, lse - M, coefficient
-    int y;
-};
-
-// one 16-byte vector of bf16 logits -> dlogits; `e0` is the column of its first element
-__device__ __forceinline__ uint4 dz_vec(uint4 z, int e0, const RowConstBf16& rc) {
-    uint32_t w[4] = {z.x, z.y, z.z, z.w};
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        float lo = ex2_approx(fmaf(bf16_lo(w[k]), kLog2e, rc.c));
-        float hi = ex2_approx(fmaf(bf16_hi(w[k]), kLog2e, rc.c));
-        uint32_t out = pack_bf16x2(lo, hi) ^ rc.sign2;
-        // the sampled token's entry is g (p_y - 1), formed in float before rounding
-        if (e0 + 2 * k == (rc.y & ~1)) {
-            const float ps = (rc.y & 1) ? hi : lo;
-            const float val = (rc.g < 0.f ? -ps : ps) - rc.g;
-            const uint32_t b = float_to_bf16_bits(val);
-            out = (rc.y & 1) ? ((out & 0x0000ffffu) | (b << 16)) : ((out & 0xffff0000u) | b);
-        }
-        w[k] = out;
-    }
-    return make_uint4(w[0], w[1], w[2], w[3]);
-}
-
-__device__ __forceinline__ uint4 dz_vec(uint4 zbits, int e0, const RowConstF32& rc) {
-    float z[4] = {__uint_as_float(zbits.x), __uint_as_float(zbits.y), __uint_as_float(zbits.z),
-                  __uint_as_float(zbits.w)};
-    uint32_t o[4];
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        float v = rc.g * expf((z[k] - rc.M) - rc.a);
-        if (e0 + k == rc.y) v -= rc.g;
-        o[k] = __float_as_uint(v);
-    }
-    return make_uint4(o[0], o[1], o[2], o[3]);
-}
-
-// scalar tail elements (vocab not a multiple of the vector width): read from the stage, written
-// straight to global memory
-__device__ __forceinline__ void dz_scalar(const void* zsm, void* orow, int e_in_chunk, int e,
-                                          const RowConstBf16& rc) {
-    const float z = __uint_as_float(((uint32_t) static_cast<const uint16_t*>(zsm)[e_in_chunk]) << 16);
-    const float ps = ex2_approx(fmaf(z, kLog2e, rc.c));
-    float val = (rc.g < 0.f) ? -ps : ps;
-    if (e == rc.y) val -= rc.g;
-    static_cast<uint16_t*>(orow)[e] = float_to_bf16_bits(val);
-}
-__device__ __forceinline__ void dz_scalar(const void* zsm, void* orow, int e_in_chunk, int e,
-                                          const RowConstF32& rc) {
-    const float z = static_cast<const float*>(zsm)[e_in_chunk];
-    float val = rc.g * expf((z - rc.M) - rc.a);
-    if (e == rc.y) val -= rc.g;
-    static_cast<float*>(orow)[e] = val;
-}
-
-// barrier over the consumer warps, returning the OR of `flag` over all of them: the decision to
-// leave after a timeout is taken by everyone together, so nobody is left waiting at a later barrier
-__device__ __forceinline__ bool consumer_barrier_or(bool flag) {
-    uint32_t out;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.u32 q, %1, 0;\n\t"
-        "bar.red.or.pred p, 1, %2, q;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(out)
-        : "r"((uint32_t)flag), "n"(kConsumers)
-        : "memory");
-    return out != 0;
-}
 
 __device__ __forceinline__ bool row_is_live(const Workspace& ws, int64_t r, int seq_len) {
     return ws.row_state[r] == ROW_OK && ws.coef[(int)(r / seq_len)] != 0.0;
@@ -279,11 +197,11 @@ dlogits_kernel(const void* logits, void* dlogits /* may alias logits */, int64_t
 #pragma unroll
                     for (int j = 0; j < kVecPerThread; ++j) {
                         const int v = tid + j * kConsumers;
-                        if (v < nv) sv[v] = dz_vec(z[j], (v0 + v) * PER, rc);
+                        if (v < nv) sv[v] = dz_vec_any(z[j], (v0 + v) * PER, rc);
                     }
                     fence_proxy_async_smem();  // generic writes above -> asynchronous read below
                 }
-                if (consumer_barrier_or(!got || *abortp != 0)) {
+                if (consumer_barrier_or<kConsumers>(!got || *abortp != 0)) {
                     ok = false;
                     break;
                 }

@@ -151,41 +151,58 @@ finalize_kernel(int n_seq, int n_groups, double eta, double norm_z, uint32_t fla
         return;
     }
 
-    // steps 3-4, one thread per group: members in index order, exactly as the definition reads
-    const bool loo = (flags & RAPID_FLAG_LEAVE_ONE_OUT) != 0;
-    for (int k = tid; k < n_groups; k += kFinThreads) {
-        const int lo = group_offsets[k], hi = group_offsets[k + 1];
-        const int Nk = hi - lo;
-        if (Nk == 0) continue;
-        double csum = 0.0;
-        for (int n = lo; n < hi; ++n) {
-            const double w = weight_of(slr, n, flags);
-            const double c = clip_w(w, eta);
-            if (full) {
-                ws.weight[n] = w;
-                ws.clipped_w[n] = c;
-            }
-            if (clipped_out) clipped_out[n] = c;
-            csum = __dadd_rn(csum, __dmul_rn(c, (double)rewards[n]));
+    // step 3, one thread per generation: the weight and its clipped value
+    for (int n = tid; n < n_seq; n += kFinThreads) {
+        const double w = weight_of(slr, n, flags);
+        const double c = clip_w(w, eta);
+        if (full) {
+            ws.weight[n] = w;
+            ws.clipped_w[n] = c;
         }
-        for (int n = lo; n < hi; ++n) {
-            double a;
-            const double R = (double)rewards[n];
-            if (loo) {
-                double others = 0.0;
-                for (int q = lo; q < hi; ++q)
-                    if (q != n)
-                        others = __dadd_rn(
-                            others, __dmul_rn(clip_w(weight_of(slr, q, flags), eta), (double)rewards[q]));
-                if (flags & RAPID_FLAG_LOO_LITERAL_DIVISOR)
-                    a = __dsub_rn(R, __ddiv_rn(others, (double)Nk));
-                else if (Nk > 1)
-                    a = __dsub_rn(R, __ddiv_rn(others, (double)(Nk - 1)));
-                else
-                    a = R;
-            } else {
-                a = __dsub_rn(R, __ddiv_rn(csum, (double)Nk));
+        if (clipped_out) clipped_out[n] = c;
+    }
+    __syncthreads();
+    auto clipped = [&](int q) -> double {
+        if (full) return ws.clipped_w[q];
+        return clipped_out ? clipped_out[q] : clip_w(weight_of(slr, q, flags), eta);
+    };
+    // step 4: every sum runs over the group's members in index order, exactly as the definition reads
+    if (!(flags & RAPID_FLAG_LEAVE_ONE_OUT)) {
+        // one thread per group: the baseline is shared by its members
+        for (int k = tid; k < n_groups; k += kFinThreads) {
+            const int lo = group_offsets[k], hi = group_offsets[k + 1];
+            const int Nk = hi - lo;
+            if (Nk == 0) continue;
+            double csum = 0.0;
+            for (int n = lo; n < hi; ++n) csum = __dadd_rn(csum, __dmul_rn(clipped(n), (double)rewards[n]));
+            const double base = __ddiv_rn(csum, (double)Nk);
+            for (int n = lo; n < hi; ++n) {
+                const double a = __dsub_rn((double)rewards[n], base);
+                if (full) ws.adv[n] = a;
+                if (adv_out) adv_out[n] = (float)a;
             }
+        }
+    } else {
+        // leave-one-out: every member has its own sum over the others, so one thread per MEMBER (a
+        // single group of thousands of generations -- the single-path baseline -- would otherwise
+        // leave N_k^2 additions to one thread).  The member's group is found by bisection.
+        for (int n = tid; n < n_seq; n += kFinThreads) {
+            int a0 = 0, a1 = n_groups;  // the last k with group_offsets[k] <= n; empty groups before it are skipped
+            while (a1 - a0 > 1) {
+                const int mid = (a0 + a1) >> 1;
+                if (group_offsets[mid] <= n) a0 = mid;
+                else a1 = mid;
+            }
+            const int lo = group_offsets[a0], hi = group_offsets[a0 + 1];
+            const int Nk = hi - lo;
+            const double R = (double)rewards[n];
+            double others = 0.0;
+            for (int q = lo; q < hi; ++q)
+                if (q != n) others = __dadd_rn(others, __dmul_rn(clipped(q), (double)rewards[q]));
+            double a;
+            if (flags & RAPID_FLAG_LOO_LITERAL_DIVISOR) a = __dsub_rn(R, __ddiv_rn(others, (double)Nk));
+            else if (Nk > 1) a = __dsub_rn(R, __ddiv_rn(others, (double)(Nk - 1)));
+            else a = R;
             if (full) ws.adv[n] = a;
             if (adv_out) adv_out[n] = (float)a;
         }

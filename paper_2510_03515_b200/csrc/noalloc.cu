@@ -5,10 +5,10 @@
 // The array's name is usable directly only in device code.  In host code the name is a host-side
 // handle, NOT a device address: handing it to a kernel would make the kernel fault (or, on
 // systems where the GPU can reach host memory, quietly scribble over the wrong bytes).  The host
-// therefore asks the runtime for the array's device address, once per device, and passes that
-// pointer on.
-#include <mutex>
-
+// therefore asks the runtime for the array's device address, with the caller's device current, and
+// passes that pointer on.  The address is asked for on EVERY call and never remembered: after the
+// first call on a device the query is a host-side table look-up, and an address remembered across a
+// cudaDeviceReset, or used under another context on the same device ordinal, would be stale.
 #include "rapid_common.cuh"
 
 namespace {
@@ -16,25 +16,14 @@ namespace {
 // One array per device that loads the library, held until the process exits.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[RAPID_NOALLOC_SCRATCH_BYTES];
 
-constexpr int kMaxDevices = 64;
-void* g_scratch_addr[kMaxDevices] = {};  // device address of the array, per device ordinal
-std::mutex g_scratch_mutex;
-
-// Device address of the scratch array on the CURRENT device; looked up on first use.
+// Device address of the scratch array on the CURRENT device.
 rapid_status_t scratch_for_current_device(void** out) {
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess) return RAPID_ERR_CUDA;
-    if (dev < 0 || dev >= kMaxDevices) return RAPID_ERR_UNSUPPORTED;
-    std::lock_guard<std::mutex> lock(g_scratch_mutex);
-    if (!g_scratch_addr[dev]) {
-        void* ptr = nullptr;
-        if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) {
-            (void)cudaGetLastError();  // leave no sticky-looking error behind for the caller
-            return RAPID_ERR_CUDA;
-        }
-        g_scratch_addr[dev] = ptr;
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) {
+        (void)cudaGetLastError();  // leave no sticky-looking error behind for the caller
+        return RAPID_ERR_CUDA;
     }
-    *out = g_scratch_addr[dev];
+    *out = ptr;
     return RAPID_OK;
 }
 

@@ -21,6 +21,7 @@
 //
 // Every wait on a barrier is bounded; a wait that gives up raises RAPID_ERR_TIMEOUT in the
 // statistics block and never traps.
+#include "dz_rows.cuh"
 #include "rapid_common.cuh"
 #include "tma_pipe.cuh"
 
@@ -41,7 +42,7 @@ namespace {
 #define RAPID_OP_HINTS 3  // see policy_evict_last() below; 3 measured best by a small margin
 #endif
 #ifndef RAPID_OP_F32X2
-#define RAPID_OP_F32X2 1  // packed two-float arithmetic in the bf16 sweeps
+#define RAPID_OP_F32X2 1  // packed two-float arithmetic in the first sweep (bf16)
 #endif
 #ifndef RAPID_OP_MINBLOCKS
 #define RAPID_OP_MINBLOCKS 2
@@ -104,22 +105,6 @@ __device__ __forceinline__ void bulk_store_hint(void* gdst, const void* smem_src
 __device__ __forceinline__ void consumer_barrier() {
     asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory");
 }
-// the same barrier, returning the OR of `flag` over all consumers: a uniform decision to leave
-__device__ __forceinline__ bool consumer_barrier_or(bool flag) {
-    uint32_t out;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.u32 q, %1, 0;\n\t"
-        "bar.red.or.pred p, 1, %2, q;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(out)
-        : "r"((uint32_t)flag), "n"(kConsumers)
-        : "memory");
-    return out != 0;
-}
-
-__device__ __forceinline__ uint16_t to_bf16_bits(float x) { return (uint16_t)(pack_bf16x2(x, 0.f) & 0xffffu); }
-
 // ---- before the pass: Eq. 2 advantages and coefficients ------------------------------------------------
 
 __global__ void __launch_bounds__(kPrepThreads)
@@ -178,34 +163,46 @@ onpolicy_prep_kernel(int n_seq, int seq_len, int vocab, int n_groups, double nor
     const double Z = (flags & RAPID_FLAG_NORM_GIVEN)    ? norm_z
                      : (flags & RAPID_FLAG_NORM_TOKENS) ? (double)tok
                                                         : (double)n_seq;
-    const bool loo = (flags & RAPID_FLAG_LEAVE_ONE_OUT) != 0;
-    // one thread per group, members in index order: the plain definition of Eq. 2
-    for (int k = tid; k < n_groups; k += kPrepThreads) {
-        const int lo = group_offsets[k], hi = group_offsets[k + 1];
-        const int Nk = hi - lo;
-        if (Nk == 0) continue;
-        double sum = 0.0;
-        for (int n = lo; n < hi; ++n) sum = __dadd_rn(sum, (double)rewards[n]);
-        for (int n = lo; n < hi; ++n) {
-            const double R = (double)rewards[n];
-            double a;
-            if (loo) {
-                double others = 0.0;
-                for (int q = lo; q < hi; ++q)
-                    if (q != n) others = __dadd_rn(others, (double)rewards[q]);
-                if (flags & RAPID_FLAG_LOO_LITERAL_DIVISOR) a = __dsub_rn(R, __ddiv_rn(others, (double)Nk));
-                else if (Nk > 1) a = __dsub_rn(R, __ddiv_rn(others, (double)(Nk - 1)));
-                else a = R;
-            } else {
-                a = __dsub_rn(R, __ddiv_rn(sum, (double)Nk));
+    auto publish = [&](int n, double a) {
+        const double g = (Z > 0.0) ? a / Z : 0.0;
+        ws.adv[n] = a;
+        ws.coef[n] = g;
+        ws.coef_log2[n] = (g != 0.0) ? log2(fabs(g)) : -INFINITY;
+        ws.weight[n] = 1.0;
+        ws.clipped_w[n] = 1.0;
+        if (adv_out) adv_out[n] = (float)a;
+    };
+    if (!(flags & RAPID_FLAG_LEAVE_ONE_OUT)) {
+        // one thread per group, members in index order: the plain definition of Eq. 2
+        for (int k = tid; k < n_groups; k += kPrepThreads) {
+            const int lo = group_offsets[k], hi = group_offsets[k + 1];
+            const int Nk = hi - lo;
+            if (Nk == 0) continue;
+            double sum = 0.0;
+            for (int n = lo; n < hi; ++n) sum = __dadd_rn(sum, (double)rewards[n]);
+            const double base = __ddiv_rn(sum, (double)Nk);
+            for (int n = lo; n < hi; ++n) publish(n, __dsub_rn((double)rewards[n], base));
+        }
+    } else {
+        // leave-one-out: one thread per member, its own index-order sum over the others of its group
+        for (int n = tid; n < n_seq; n += kPrepThreads) {
+            int a0 = 0, a1 = n_groups;  // the last k with group_offsets[k] <= n
+            while (a1 - a0 > 1) {
+                const int mid = (a0 + a1) >> 1;
+                if (group_offsets[mid] <= n) a0 = mid;
+                else a1 = mid;
             }
-            const double g = (Z > 0.0) ? a / Z : 0.0;
-            ws.adv[n] = a;
-            ws.coef[n] = g;
-            ws.coef_log2[n] = (g != 0.0) ? log2(fabs(g)) : -INFINITY;
-            ws.weight[n] = 1.0;
-            ws.clipped_w[n] = 1.0;
-            if (adv_out) adv_out[n] = (float)a;
+            const int lo = group_offsets[a0], hi = group_offsets[a0 + 1];
+            const int Nk = hi - lo;
+            const double R = (double)rewards[n];
+            double others = 0.0;
+            for (int q = lo; q < hi; ++q)
+                if (q != n) others = __dadd_rn(others, (double)rewards[q]);
+            double a;
+            if (flags & RAPID_FLAG_LOO_LITERAL_DIVISOR) a = __dsub_rn(R, __ddiv_rn(others, (double)Nk));
+            else if (Nk > 1) a = __dsub_rn(R, __ddiv_rn(others, (double)(Nk - 1)));
+            else a = R;
+            publish(n, a);
         }
     }
     if (tid == 0) {
@@ -215,17 +212,6 @@ onpolicy_prep_kernel(int n_seq, int seq_len, int vocab, int n_groups, double nor
 }
 
 // ---- the pass ------------------------------------------------------------------------------------------
-
-struct RowConstBf16 {
-    float c;         // -lse log2(e) + log2|g|
-    float g;
-    uint32_t sign2;  // sign of g on both halves of a packed pair
-    int y;
-};
-struct RowConstF32 {
-    float M, a, g;  // row max, lse - M, coefficient
-    int y;
-};
 
 // running (max, sum of exponentials) of one thread
 struct Acc {
@@ -312,58 +298,6 @@ __device__ __forceinline__ void acc_scalar(Acc& a, float z, bool base2) {
         a.m = z;
     }
     a.s0 += base2 ? ex2_approx((z - a.m) * kLog2e) : expf(z - a.m);
-}
-
-template <bool HAS_Y>
-__device__ __forceinline__ uint4 dz_vec(uint4 z, int e0, const RowConstBf16& rc) {
-    uint32_t w[4] = {z.x, z.y, z.z, z.w};
-#if RAPID_OP_F32X2
-    const uint64_t k2 = f32x2(kLog2e, kLog2e), c2 = f32x2(rc.c, rc.c);
-#endif
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-#if RAPID_OP_F32X2
-        float xl, xh;
-        f32x2_split(f32x2_fma(f32x2(bf16_lo(w[k]), bf16_hi(w[k])), k2, c2), xl, xh);
-        const float lo = ex2_approx(xl), hi = ex2_approx(xh);
-#else
-        const float lo = ex2_approx(fmaf(bf16_lo(w[k]), kLog2e, rc.c));
-        const float hi = ex2_approx(fmaf(bf16_hi(w[k]), kLog2e, rc.c));
-#endif
-        uint32_t out = pack_bf16x2(lo, hi) ^ rc.sign2;
-        if (HAS_Y && e0 + 2 * k == (rc.y & ~1)) {  // the sampled token: g (p_y - 1), formed in float
-            const float ps = (rc.y & 1) ? hi : lo;
-            const uint32_t b = to_bf16_bits((rc.g < 0.f ? -ps : ps) - rc.g);
-            out = (rc.y & 1) ? ((out & 0x0000ffffu) | (b << 16)) : ((out & 0xffff0000u) | b);
-        }
-        w[k] = out;
-    }
-    return make_uint4(w[0], w[1], w[2], w[3]);
-}
-template <bool HAS_Y>
-__device__ __forceinline__ uint4 dz_vec(uint4 zb, int e0, const RowConstF32& rc) {
-    const float z[4] = {__uint_as_float(zb.x), __uint_as_float(zb.y), __uint_as_float(zb.z), __uint_as_float(zb.w)};
-    uint32_t o[4];
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        float v = rc.g * expf((z[k] - rc.M) - rc.a);
-        if (HAS_Y && e0 + k == rc.y) v -= rc.g;
-        o[k] = __float_as_uint(v);
-    }
-    return make_uint4(o[0], o[1], o[2], o[3]);
-}
-__device__ __forceinline__ void dz_scalar(const void* zsm, void* orow, int e_in_chunk, int e, const RowConstBf16& rc) {
-    const float z = __uint_as_float(((uint32_t) static_cast<const uint16_t*>(zsm)[e_in_chunk]) << 16);
-    const float ps = ex2_approx(fmaf(z, kLog2e, rc.c));
-    float val = (rc.g < 0.f) ? -ps : ps;
-    if (e == rc.y) val -= rc.g;
-    static_cast<uint16_t*>(orow)[e] = to_bf16_bits(val);
-}
-__device__ __forceinline__ void dz_scalar(const void* zsm, void* orow, int e_in_chunk, int e, const RowConstF32& rc) {
-    const float z = static_cast<const float*>(zsm)[e_in_chunk];
-    float val = rc.g * expf((z - rc.M) - rc.a);
-    if (e == rc.y) val -= rc.g;
-    static_cast<float*>(orow)[e] = val;
 }
 
 // Which sweeps a row gets.  Decided from the inputs alone, identically by every thread.
@@ -640,7 +574,7 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
                     sh_m[warp] = wm;
                     sh_s[warp] = (double)sm;
                 }
-                if (consumer_barrier_or(!ok || *abortp != 0)) {
+                if (consumer_barrier_or<kConsumers>(!ok || *abortp != 0)) {
                     ok = false;
                     break;
                 }
@@ -709,8 +643,7 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
                     for (int j = 0; j < kVecPerThread; ++j) {
                         const int e = e0 + j * 32 * PER;
                         // the sampled token's column is looked for once per vector, not once per element
-                        wv[j * 32] = ((unsigned)(rc.y - e) < (unsigned)PER) ? dz_vec<true>(z[j], e, rc)
-                                                                            : dz_vec<false>(z[j], e, rc);
+                        wv[j * 32] = dz_vec_any(z[j], e, rc);
                     }
                 } else {
 #pragma unroll

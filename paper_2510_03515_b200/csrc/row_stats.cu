@@ -46,34 +46,33 @@ struct FloatSum {
     __device__ __forceinline__ double value() const { return (double)s + (double)c; }
 };
 
-// A thread's state is (m, sh, S, T): the largest logit seen, the shift sh = ceil(fl(m k)) with
-// k = fl(log2 e) that its exponentials were taken against (an integer, so that moving to a new shift
-// multiplies by an exact power of two) plus a 16-bit fraction `off` that differs from thread to
-// thread, S = sum_v e_v with e_v = 2^(x_v), x_v = z_v k - sh, and
-// T = sum_v x_v e_v.  Three things keep the log-sum-exp free of any bias beyond a few 1e-9, which a
-// generation-level weight multiplies by the generation's length:
-//  * the shift is USED as it stands, in the exponentials and again when threads are combined, and
-//    turned back into natural-log units as sh / k, so no rounding of m k enters;
-//  * k differs from log2(e) by rho = 1.3e-8 (relative), so the wanted term is 2^(x (1 + rho)) =
-//    e_v (1 + rho ln2 x_v): the first-order correction rho ln2 T is added to S at the end;
+// A thread's state is (m, sh, S): the largest logit seen, the shift sh that its exponentials were taken
+// against, and S = sum_v 2^(x_v) with x_v = z_v log2(e) - sh.  A generation-level weight multiplies
+// any bias of the token log-probs by the generation's length, so four things keep the log-sum-exp
+// free of bias beyond about 1e-9:
+//  * sh = ceil(m log2 e) + off is USED as it stands, in the exponentials and again when threads are
+//    combined (in double), so no rounding of m log2(e) enters.  Its integer part makes moving to a new
+//    shift a multiplication by an exact power of two.
+//  * log2(e) is applied as kK1 + kK2: kK1 has 16 significant bits, so its product with a bf16 logit
+//    (8 bits) is exact, and the float kK2 carries the next 24 bits.  A single float constant is off by
+//    1.3e-8 relative, which shifts the log-sum-exp by that times the softmax-weighted mean distance
+//    below the shift: 5e-8 for these logits.
 //  * the hardware exponential's relative error on negative arguments, averaged over the fraction of
 //    the argument, is kEx2Bias (measured over all 2^23 fractions on sm_100a: -5.0e-8, the same to 3 %
 //    for every integer part; errors lie in [-1.44e-7, +0.63e-7]); a sum of many terms carries that
-//    mean, and is divided by 1 + kEx2Bias.  bf16 logits take few distinct values and k is fixed, so
-//    with a common integer shift the fraction of x_v would depend on z_v alone and the sum would carry
-//    the errors of those few fractions (a bias of 1e-8 either way) instead of the mean; the per-thread
-//    fraction of the shift spreads every logit value over 128 different fractions.
+//    mean, and is divided by 1 + kEx2Bias.  bf16 logits take few distinct values, so with a common
+//    integer shift the fraction of x_v would depend on z_v alone and the sum would carry the errors of
+//    those few fractions (1e-8 either way) instead of the mean; the 16-bit fraction `off`, different
+//    for every thread, spreads each logit value over 128 fractions.
 //  * the thread's largest logit, which may carry nearly all of the row's probability, gets no such
-//    statistical treatment: its hardware exponential is taken out of S and T again at the end of the
-//    sweep and replaced by the exact value in double.
+//    statistical treatment: its hardware exponential is taken out of S again at the end of the sweep
+//    and replaced by the exact value in double.
 constexpr float kEx2Bias = -5.0e-8f;
-constexpr double kLog2eF = (double)kLog2e;                       // the float constant, exactly
-constexpr double kOnePlusRho = kLog2eD / kLog2eF;
-constexpr double kRhoLn2 = (kLog2eD - kLog2eF) / kLog2eF * kLn2D;  // rho ln 2
+constexpr float kK1 = 47274.f / 32768.f;                   // log2(e) rounded down to 16 bits
+constexpr float kK2 = (float)(kLog2eD - 47274.0 / 32768.0);  // > 0, so that -inf logits stay -inf
 
 template <int U>
-__device__ __forceinline__ void bf16_batch(const uint4 (&q)[U], float off, float& m, float& sh, FloatSum& S,
-                                           float& T) {
+__device__ __forceinline__ void bf16_batch(const uint4 (&q)[U], float off, float& m, float& sh, FloatSum& S) {
     uint32_t mx = bf16x2_max(bf16x2_max(q[0].x, q[0].y), bf16x2_max(q[0].z, q[0].w));
 #pragma unroll
     for (int j = 1; j < U; ++j)
@@ -86,36 +85,27 @@ __device__ __forceinline__ void bf16_batch(const uint4 (&q)[U], float off, float
         m = bm;
         if (bm > -1.0e38f) {
             const float nsh = ceilf(bm * kLog2e) + off;
-            const float f = ex2_approx(sh - nsh);  // exact: an integer power of two (and S = T = 0 for an empty thread)
-            T = f * fmaf(sh - nsh, S.s, T);        // every x moves by sh - nsh
-            S.scale(f);
+            S.scale(ex2_approx(sh - nsh));  // an exact power of two (S is still 0 for an empty thread's shift 0)
             sh = nsh;
         }
     }
     // a pair of logits at a time in the packed two-float forms (one instruction for two multiply-adds
-    // or two additions, each rounded like its scalar form).  Masked entries (-inf, or the lowest finite
-    // value) are raised to -1e30 first: their exponential is still exactly 0, and 0 * x stays 0 in T.
-    const uint64_t k2 = f32x2(kLog2e, kLog2e), nsh2 = f32x2(-sh, -sh);
-    constexpr uint32_t kFloor2 = 0xf14af14au;  // bf16 pair (-1.0e30, -1.0e30)
-    uint64_t s2 = f32x2(0.f, 0.f), t2 = f32x2(0.f, 0.f);
+    // or two additions, each rounded like its scalar form)
+    const uint64_t k1 = f32x2(kK1, kK1), k2 = f32x2(kK2, kK2), nsh2 = f32x2(-sh, -sh);
+    uint64_t s2 = f32x2(0.f, 0.f);
 #pragma unroll
     for (int j = 0; j < U; ++j) {
         const uint32_t w[4] = {q[j].x, q[j].y, q[j].z, q[j].w};
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            const uint32_t z2 = bf16x2_max(w[k], kFloor2);
-            const uint64_t x2 = f32x2_fma(f32x2(bf16_lo(z2), bf16_hi(z2)), k2, nsh2);
+            const uint64_t z2 = f32x2(bf16_lo(w[k]), bf16_hi(w[k]));
             float x0, x1;
-            f32x2_split(x2, x0, x1);
-            const uint64_t e2 = f32x2(ex2_approx(x0), ex2_approx(x1));
-            s2 = f32x2_add(s2, e2);
-            t2 = f32x2_fma(x2, e2, t2);
+            f32x2_split(f32x2_fma(z2, k2, f32x2_fma(z2, k1, nsh2)), x0, x1);
+            s2 = f32x2_add(s2, f32x2(ex2_approx(x0), ex2_approx(x1)));
         }
     }
-    float s0, s1, t0, t1;
+    float s0, s1;
     f32x2_split(s2, s0, s1);
-    f32x2_split(t2, t0, t1);
-    T += t0 + t1;
     const float b = s0 + s1;
     if (b > S.s) {  // keep the larger operand first, as Fast2Sum wants (early batches only)
         const float old = S.s;
@@ -128,7 +118,7 @@ __device__ __forceinline__ void bf16_batch(const uint4 (&q)[U], float off, float
 
 // `out`, when not null, receives a copy of the row (same layout): used when the logits are read from
 // host memory and the second pass wants them on the device.
-// Returns the thread's maximum, its shift (log2 units) and its share of sum_v exp(z_v - sh / k), all
+// Returns the thread's maximum, its shift (log2 units) and its share of sum_v 2^(z_v log2(e) - sh), all
 // corrections applied; a thread that saw nothing real returns 0 and the shift 0.
 __device__ __forceinline__ void row_sweep_bf16(const uint16_t* row, int vocab, float& m_out, float& sh_out,
                                                double& s_out, uint16_t* out) {
@@ -137,7 +127,7 @@ __device__ __forceinline__ void row_sweep_bf16(const uint16_t* row, int vocab, f
     const int nvec = vocab >> 3;
     const uint4* rv = reinterpret_cast<const uint4*>(row);
     uint4* ov = reinterpret_cast<uint4*>(out);
-    float m = -INFINITY, sh = 0.f, T = 0.f;
+    float m = -INFINITY, sh = 0.f;
     FloatSum S{0.f, 0.f};
     // this thread's fraction of the shift (see above): 16 bits, scattered, so that the fractions neither
     // line up with a table of the hardware exponential nor cost the shift its exactness
@@ -151,16 +141,16 @@ __device__ __forceinline__ void row_sweep_bf16(const uint16_t* row, int vocab, f
 #pragma unroll
             for (int j = 0; j < U; ++j) ov[v + j * kThreads] = q[j];
         }
-        bf16_batch<U>(q, off, m, sh, S, T);
+        bf16_batch<U>(q, off, m, sh, S);
     }
     for (; v < nvec; v += kThreads) {
         uint4 q[1];
         q[0] = ld_stream(rv + v);
         if (out) ov[v] = q[0];
-        bf16_batch<1>(q, off, m, sh, S, T);
+        bf16_batch<1>(q, off, m, sh, S);
     }
     // ragged tail (vocab not a multiple of 8): one element per thread
-    double tail = 0.0, tail_t = 0.0;
+    double tail = 0.0;
     const int e = (nvec << 3) + tid;
     if (e < vocab) {
         const uint16_t zb = row[e];
@@ -170,29 +160,20 @@ __device__ __forceinline__ void row_sweep_bf16(const uint16_t* row, int vocab, f
             m = z;
             if (z > -1.0e38f) {
                 const float nsh = ceilf(z * kLog2e) + off;
-                const float f = ex2_approx(sh - nsh);
-                T = f * fmaf(sh - nsh, S.s, T);
-                S.scale(f);
+                S.scale(ex2_approx(sh - nsh));
                 sh = nsh;
             }
         }
-        if (z > -1.0e38f) {
-            const float x = fmaf(z, kLog2e, -sh);
-            tail = (double)ex2_approx(x);
-            tail_t = (double)fmaxf(x, -200.f) * tail;
-        }
+        if (z > -1.0e38f) tail = (double)ex2_approx(fmaf(z, kK2, fmaf(z, kK1, -sh)));
     }
     m_out = m;
     sh_out = sh;
-    double s = S.value() + tail, t = (double)T + tail_t, top = 0.0;
+    double s = S.value() + tail, top = 0.0;
     if (m > -1.0e38f) {  // the largest logit: out with what the hardware gave for it, in with the exact term
-        const float xm = fmaf(m, kLog2e, -sh);
-        const float em = ex2_approx(xm);
-        s -= (double)em;
-        t -= (double)xm * (double)em;
-        top = exp2(((double)m * kLog2eF - (double)sh) * kOnePlusRho);
+        s -= (double)ex2_approx(fmaf(m, kK2, fmaf(m, kK1, -sh)));
+        top = exp2((double)m * kLog2eD - (double)sh);
     }
-    s_out = (s + kRhoLn2 * t) / (1.0 + (double)kEx2Bias) + top;
+    s_out = s / (1.0 + (double)kEx2Bias) + top;
 }
 
 // ---- fp32 ------------------------------------------------------------------------------------
@@ -281,7 +262,7 @@ row_stats_kernel(const void* __restrict__ logits, void* __restrict__ copy_out, i
 
         float M;
         double S;      // the row's sum of exponentials against `shift`
-        double shift;  // M for float logits; the float shift actually used, in natural-log units, for bf16
+        double shift;  // M for float logits; the shift actually used, in natural-log units, for bf16
         double zy;
         if (DT == RAPID_BF16) {
             const uint16_t* row = static_cast<const uint16_t*>(logits) + i * ld;
@@ -293,7 +274,7 @@ row_stats_kernel(const void* __restrict__ logits, void* __restrict__ copy_out, i
             // a thread (or a whole warp, for a tiny vocabulary) that saw nothing has s = 0
             const float wm = warp_max(m);
             const float wsh = warp_max(s > 0.0 ? sh : -INFINITY);
-            if (s > 0.0 && sh != wsh) s *= exp2(((double)sh - (double)wsh) * kOnePlusRho);
+            if (s > 0.0 && sh != wsh) s *= exp2((double)sh - (double)wsh);
             s = warp_sum(s);
             if (lane == 0) {
                 sh_m[warp] = wm;
@@ -309,10 +290,10 @@ row_stats_kernel(const void* __restrict__ logits, void* __restrict__ copy_out, i
                 }
                 double tot = 0.0;
                 for (int w = 0; w < kWarps; ++w)
-                    if (sh_s[w] > 0.0) tot += sh_s[w] * exp2(((double)sh_sh[w] - (double)msh) * kOnePlusRho);
+                    if (sh_s[w] > 0.0) tot += sh_s[w] * exp2((double)sh_sh[w] - (double)msh);
                 M = mm;
                 S = tot;
-                shift = (double)msh / kLog2eF;  // lse = shift + log(S)
+                shift = (double)msh * kLn2D;  // lse = shift + log(S)
                 zy = (double)__uint_as_float(((uint32_t)row[y]) << 16);  // (one more 2-byte read of the row)
             }
         } else {

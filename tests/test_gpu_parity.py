@@ -223,6 +223,27 @@ def test_group_advantage_bit_exact(flags, eta):
         assert st["n_clipped"] == 0 and st["mean_log_cw"] == 0.0
 
 
+@pytest.mark.parametrize("flags", [0, rb.FLAG_LEAVE_ONE_OUT, rb.FLAG_LEAVE_ONE_OUT | rb.FLAG_LOO_LITERAL_DIVISOR])
+@pytest.mark.parametrize("sizes", [[3000], [5, 0, 0, 2900, 0, 7, 1, 0]])
+def test_group_advantage_groups_of_thousands(flags, sizes):
+    """The single-path baseline (every generation in one group) with thousands of generations, and the
+    same beside small and empty groups: the leave-one-out sums run one thread per member and find
+    the member's group by bisection over offsets that repeat where a group is empty.  Bit-exact."""
+    rng = np.random.default_rng(23)
+    go = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int32)
+    N = int(go[-1])
+    R = rng.normal(0, 1, N).astype(np.float32)
+    w = np.exp(rng.normal(0, 1.0, N))
+    ref = oracle.group_advantage(R, w, go, 2.0, flags | oracle.FLAG_ADV_INPUT_IS_WEIGHT)
+    adv, cw, st = _adv_gpu(R, w, go, 2.0, flags | rb.FLAG_ADV_INPUT_IS_WEIGHT)
+    assert np.array_equal(adv.view(np.uint32), ref["adv32"].view(np.uint32))
+    assert np.array_equal(cw, ref["clipped_w"]) and st["status"] == 0
+    assert st["n_empty_group"] == sizes.count(0)
+    ref = oracle.group_advantage(R, None, go, 2.0, flags)
+    adv, _, _ = _adv_gpu(R, None, go, 2.0, flags)
+    assert np.array_equal(adv.view(np.uint32), ref["adv32"].view(np.uint32))
+
+
 def test_group_advantage_zero_sum_on_device():
     """Eq. 2 advantages sum to zero within each group (checked on the device's own output)."""
     rng = np.random.default_rng(19)

@@ -166,3 +166,11 @@ def test_fused_head_argument_validation():
     assert T * ((V + 63) // 64 * 64) * 2 <= n <= T * ((V + 63) // 64 * 64) * 2 + 2 * 594 * T * 4 + 64 * T
     with pytest.raises(rb.RapidError):
         rb.rapid_fused_head_workspace_bytes(rb.make_desc(64, 256, 151936, 8, torch.float32), 1536)
+
+
+def test_bounded_wait_selftest_refuses_bad_limits_on_the_host():
+    """NULL statistics, a zero limit and a limit above one second are refused before anything is launched."""
+    L = rb.lib()
+    assert L.rapid_selftest_bounded_wait(1000, None, None) == rb.RAPID_ERR_INVALID_ARG
+    assert L.rapid_selftest_bounded_wait(0, FAKE, None) == rb.RAPID_ERR_INVALID_ARG
+    assert L.rapid_selftest_bounded_wait(1_000_000_001, FAKE, None) == rb.RAPID_ERR_UNSUPPORTED
