@@ -56,6 +56,13 @@ constexpr int kStages = RAPID_OP_STAGES;
 #define RAPID_OP_PENDING 3
 #endif
 constexpr int kMaxPending = RAPID_OP_PENDING;  // bulk stores that may still be reading their stage
+#ifndef RAPID_OP_RETAIN
+#define RAPID_OP_RETAIN 2
+#endif
+// The last kRetain chunks of a row's first sweep are not given back to the producer: they stay in their
+// stages, and the second sweep starts on them in place instead of loading them again.
+constexpr int kRetain = RAPID_OP_RETAIN;
+static_assert(kRetain >= 0 && kRetain + kMaxPending < RAPID_OP_STAGES, "retained stages, stages that pending stores hold and one to load into");
 static_assert(kStages >= kMaxPending + 2, "the ring must keep cycling while stores are in flight");
 static_assert((kChunk / 16) % kConsumers == 0, "a chunk is a whole number of 16-byte vectors per consumer");
 constexpr int kVecPerChunk = kChunk / 16;
@@ -395,7 +402,9 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
                 for (int sweep = 0; sweep < plan && ok; ++sweep) {
                     // first sweep of a row that will be read again: ask L2 to keep it
                     const uint64_t pol = (sweep == 0 && plan == ROWS_BOTH) ? keep : stream;
-                    for (int c = 0; c < n_chunks; ++c, ++it) {
+                    // the second sweep finds the row's last chunks still in shared memory
+                    const int n_load = (sweep == 1) ? n_chunks - min(kRetain, n_chunks) : n_chunks;
+                    for (int c = 0; c < n_load; ++c, ++it) {
                         const int s = it % kStages;
                         const uint32_t use = it / kStages;
                         if (use > 0 && !mbar_wait_bounded(&empty_bar[s], (use & 1u) ^ 1u, abortp)) {
@@ -509,9 +518,12 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
             // chunk and gives the stage back on its own (the stage's barrier counts the warps), so no
             // CTA-wide barrier is needed per chunk ----
             Acc acc{-INFINITY, 0.f, 0.f};
+            const int n_ret = (plan == ROWS_BOTH) ? min(kRetain, n_chunks) : 0;  // chunks kept for the second sweep
+            int ret_st = 0;                                                     // stage of the first of them
             if (ok) {
                 for (int c = 0; c < n_chunks; ++c) {
                     const int s = st;
+                    if (c == n_chunks - n_ret) ret_st = s;
                     const bool got = mbar_wait_bounded(&full_bar[s], ph, abortp);
                     if (__any_sync(0xffffffffu, !got)) {
                         ok = false;
@@ -554,9 +566,9 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
                     if (tid == 0 && yi >= 0 && yi < kVecPerChunk * PER)
                         sh_zy = (ESIZE == 2) ? __uint_as_float(((uint32_t) reinterpret_cast<const uint16_t*>(sv)[yi]) << 16)
                                              : reinterpret_cast<const float*>(sv)[yi];
-                    __syncwarp();  // the whole warp has its data in registers: the stage can go
+                    __syncwarp();  // the whole warp has its data in registers: the stage can go (unless it is kept)
                     if (lane == 0) {
-                        mbar_arrive(&empty_bar[s]);
+                        if (c < n_chunks - n_ret) mbar_arrive(&empty_bar[s]);
                         if (c < kMaxPending) drain_one();  // stages still held by this warp's stores of the previous row
                     }
                     if (full) acc_vec<true>(acc, q, kVecPerThread, (RowConst*)nullptr);
@@ -617,14 +629,8 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
                 rc.g = (float)g;
                 rc.y = y;
             }
-            for (int c = 0; c < n_chunks && ok; ++c) {
-                const int s = st;
-                const bool got = mbar_wait_bounded(&full_bar[s], ph, abortp);
-                if (__any_sync(0xffffffffu, !got)) {
-                    ok = false;
-                    break;
-                }
-                next_stage();
+            // chunk c of the row sits in stage s: dlogits in place, then out
+            auto second_sweep_chunk = [&](int c, int s) {
                 uint4* sv = reinterpret_cast<uint4*>(ring + (size_t)s * kChunk);
                 const int v0 = c * kVecPerChunk;
                 const int nv = min(kVecPerChunk, nvec_row - v0);
@@ -663,6 +669,23 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
                         mbar_arrive(&empty_bar[s]);  // nothing to send from this slice
                     }
                 }
+            };
+            {   // first the chunks kept from the first sweep, where they lie
+                int rs = ret_st;
+                for (int c = n_chunks - n_ret; c < n_chunks; ++c) {
+                    second_sweep_chunk(c, rs);
+                    if (++rs == kStages) rs = 0;
+                }
+            }
+            for (int c = 0; c < n_chunks - n_ret && ok; ++c) {
+                const int s = st;
+                const bool got = mbar_wait_bounded(&full_bar[s], ph, abortp);
+                if (__any_sync(0xffffffffu, !got)) {
+                    ok = false;
+                    break;
+                }
+                next_stage();
+                second_sweep_chunk(c, s);
             }
         }
         // a warp that gave up in the middle of a row still owes nothing to a barrier: the others see

@@ -34,6 +34,7 @@ struct Workspace {
     int32_t* seq_tokens;    // [N]
     int32_t* seq_bad;       // [N] rows with a target id outside [0, V)
     rapid_stats_t* stats;   // [1]
+    unsigned int* row_ticket;  // [1] next row of the statistics pass (zeroed by each launch)
 };
 
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -64,6 +65,7 @@ __host__ inline size_t carve_workspace(const rapid_desc_t& d, void* base, Worksp
     ws.seq_tokens = reinterpret_cast<int32_t*>(take(N * 4));
     ws.seq_bad = reinterpret_cast<int32_t*>(take(N * 4));
     ws.stats = reinterpret_cast<rapid_stats_t*>(take(sizeof(rapid_stats_t)));
+    ws.row_ticket = reinterpret_cast<unsigned int*>(take(sizeof(unsigned int)));
     if (w) *w = ws;
     return off;
 }

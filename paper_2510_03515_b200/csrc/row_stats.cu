@@ -15,13 +15,17 @@ namespace rapid {
 namespace {
 
 #ifndef RAPID_P1_THREADS
-#define RAPID_P1_THREADS 128
+#define RAPID_P1_THREADS 128  // bf16 logits
+#endif
+#ifndef RAPID_P1_THREADS_F32
+#define RAPID_P1_THREADS_F32 128  // float logits
 #endif
 #ifndef RAPID_P1_U
 #define RAPID_P1_U 8  // 16-byte loads in flight per thread (bf16 sweep)
 #endif
-constexpr int kThreads = RAPID_P1_THREADS;
-constexpr int kWarps = kThreads / 32;
+#ifndef RAPID_P1_TICKETS
+#define RAPID_P1_TICKETS 1  // rows handed out through a counter (1) or grid-stride (0)
+#endif
 
 // ---- bf16 ------------------------------------------------------------------------------------
 
@@ -120,6 +124,7 @@ __device__ __forceinline__ void bf16_batch(const uint4 (&q)[U], float off, float
 // host memory and the second pass wants them on the device.
 // Returns the thread's maximum, its shift (log2 units) and its share of sum_v 2^(z_v log2(e) - sh), all
 // corrections applied; a thread that saw nothing real returns 0 and the shift 0.
+template <int kThreads>
 __device__ __forceinline__ void row_sweep_bf16(const uint16_t* row, int vocab, float& m_out, float& sh_out,
                                                double& s_out, uint16_t* out) {
     constexpr int U = RAPID_P1_U;
@@ -194,6 +199,7 @@ __device__ __forceinline__ void f32_batch(const float4* q, int n, float& m, doub
         s += (double)((expf(q[j].x - m) + expf(q[j].y - m)) + (expf(q[j].z - m) + expf(q[j].w - m)));
 }
 
+template <int kThreads>
 __device__ __forceinline__ void row_sweep_f32(const float* row, int vocab, float& m_out, double& s_out,
                                               float* out) {
     constexpr int U = 4;
@@ -236,17 +242,29 @@ __device__ __forceinline__ void row_sweep_f32(const float* row, int vocab, float
 
 // ---- kernel ----------------------------------------------------------------------------------
 
-template <int DT>
+// Rows are handed out one at a time through a counter (`ticket`, zero at launch) when one is given, so
+// that every CTA stays busy until the rows run out whatever the pattern of masked rows; without a counter
+// CTA b takes rows b, b + grid, ...
+template <int DT, int kThreads>
 __global__ void __launch_bounds__(kThreads)
 row_stats_kernel(const void* __restrict__ logits, void* __restrict__ copy_out, int64_t ld, int vocab, int64_t row0,
                  int64_t n_rows, const int32_t* __restrict__ targets,
-                 const uint8_t* __restrict__ mask, Workspace ws) {
+                 const uint8_t* __restrict__ mask, unsigned int* ticket, Workspace ws) {
+    constexpr int kWarps = kThreads / 32;
     __shared__ float sh_m[kWarps];
     __shared__ float sh_sh[kWarps];
     __shared__ double sh_s[kWarps];
+    __shared__ unsigned int sh_next;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-    for (int64_t i = blockIdx.x; i < n_rows; i += gridDim.x) {
+    for (int64_t i = blockIdx.x;; i += gridDim.x) {
+        if (ticket) {  // uniform
+            if (tid == 0) sh_next = atomicAdd(ticket, 1u);
+            __syncthreads();
+            i = sh_next;
+            __syncthreads();  // everyone has read it before thread 0 draws again
+        }
+        if (i >= n_rows) break;
         const int64_t r = row0 + i;
         const bool on = mask ? (mask[r] != 0) : true;
         const int32_t y = targets[r];
@@ -269,7 +287,7 @@ row_stats_kernel(const void* __restrict__ logits, void* __restrict__ copy_out, i
             float m, sh;
             double s;
             uint16_t* orow = copy_out ? static_cast<uint16_t*>(copy_out) + i * ld : nullptr;
-            row_sweep_bf16(row, vocab, m, sh, s, orow);
+            row_sweep_bf16<kThreads>(row, vocab, m, sh, s, orow);
             // threads are brought to a common shift in double, with the shifts exactly as they were used;
             // a thread (or a whole warp, for a tiny vocabulary) that saw nothing has s = 0
             const float wm = warp_max(m);
@@ -301,7 +319,7 @@ row_stats_kernel(const void* __restrict__ logits, void* __restrict__ copy_out, i
             float m;
             double s;
             float* orow = copy_out ? static_cast<float*>(copy_out) + i * ld : nullptr;
-            row_sweep_f32(row, vocab, m, s, orow);
+            row_sweep_f32<kThreads>(row, vocab, m, s, orow);
             const float wm = warp_max(m);
             // a thread that saw nothing has m = -inf and s = 0
             double sd = (s > 0.0) ? s * exp((double)m - (double)wm) : 0.0;
@@ -336,29 +354,36 @@ row_stats_kernel(const void* __restrict__ logits, void* __restrict__ copy_out, i
 
 }  // namespace
 
-cudaError_t launch_row_stats(const rapid_desc_t& d, const void* logits_chunk, int64_t row0,
-                             int64_t n_rows, const int32_t* targets, const uint8_t* mask,
-                             const Workspace& ws, int sm_count, cudaStream_t stream, void* copy_out) {
-    if (n_rows <= 0) return cudaSuccess;
+template <int DT, int kThreads>
+static cudaError_t launch_one(const rapid_desc_t& d, const void* logits_chunk, int64_t row0, int64_t n_rows,
+                              const int32_t* targets, const uint8_t* mask, const Workspace& ws, int sm_count,
+                              cudaStream_t stream, void* copy_out) {
     int per_sm = 0;
-    cudaError_t e;
-    if (d.dtype == RAPID_BF16)
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, row_stats_kernel<RAPID_BF16>,
-                                                          kThreads, 0);
-    else
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, row_stats_kernel<RAPID_F32>,
-                                                          kThreads, 0);
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, row_stats_kernel<DT, kThreads>, kThreads, 0);
     if (e != cudaSuccess) return e;
     if (per_sm < 1) per_sm = 1;
     int64_t grid = (int64_t)sm_count * per_sm;
     if (grid > n_rows) grid = n_rows;
-    if (d.dtype == RAPID_BF16)
-        row_stats_kernel<RAPID_BF16><<<(unsigned)grid, kThreads, 0, stream>>>(
-            logits_chunk, copy_out, d.ld, d.vocab, row0, n_rows, targets, mask, ws);
-    else
-        row_stats_kernel<RAPID_F32><<<(unsigned)grid, kThreads, 0, stream>>>(
-            logits_chunk, copy_out, d.ld, d.vocab, row0, n_rows, targets, mask, ws);
+    unsigned int* ticket = RAPID_P1_TICKETS ? ws.row_ticket : nullptr;
+    if (ticket) {
+        e = cudaMemsetAsync(ticket, 0, sizeof(unsigned int), stream);
+        if (e != cudaSuccess) return e;
+    }
+    row_stats_kernel<DT, kThreads><<<(unsigned)grid, kThreads, 0, stream>>>(logits_chunk, copy_out, d.ld, d.vocab, row0,
+                                                                           n_rows, targets, mask, ticket, ws);
     return cudaGetLastError();
+}
+
+cudaError_t launch_row_stats(const rapid_desc_t& d, const void* logits_chunk, int64_t row0,
+                             int64_t n_rows, const int32_t* targets, const uint8_t* mask,
+                             const Workspace& ws, int sm_count, cudaStream_t stream, void* copy_out) {
+    if (n_rows <= 0) return cudaSuccess;
+    if (n_rows > 0xffffffffll) return cudaErrorInvalidValue;  // the row counter is 32 bits wide
+    if (d.dtype == RAPID_BF16)
+        return launch_one<RAPID_BF16, RAPID_P1_THREADS>(d, logits_chunk, row0, n_rows, targets, mask, ws, sm_count,
+                                                        stream, copy_out);
+    return launch_one<RAPID_F32, RAPID_P1_THREADS_F32>(d, logits_chunk, row0, n_rows, targets, mask, ws, sm_count,
+                                                       stream, copy_out);
 }
 
 }  // namespace rapid

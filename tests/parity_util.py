@@ -13,9 +13,14 @@ from paper_2510_03515_b200 import synth
 
 LOSS_RTOL = {torch.float32: 1e-5, torch.bfloat16: 2e-3}
 DLOGITS_ATOL = {torch.float32: 1e-6, torch.bfloat16: 4e-3}
-# token log-probs are returned as float32: half an ulp at |x| ~ 16 is 1e-6
-LOGP_ATOL = {torch.float32: 2e-6, torch.bfloat16: 2e-5}
-ADV_ATOL = {torch.float32: 2e-6, torch.bfloat16: 2e-4}
+# token log-probs are returned as float32: half an ulp at |x| in [16, 32) is 1e-6, which is what is
+# observed (worst 9.6e-7 at full size); the kernels' own error is below 2e-7
+LOGP_ATOL = {torch.float32: 2e-6, torch.bfloat16: 4e-6}
+ADV_ATOL = {torch.float32: 2e-6, torch.bfloat16: 2e-5}
+# the fused LM-head form takes its row statistics in float inside the GEMM epilogue, 256 columns at a
+# time (observed at full size: token log-probs 7e-6, advantages 1.8e-5)
+HEAD_LOGP_ATOL = 2e-5
+HEAD_ADV_ATOL = 2e-4
 
 
 def report_observed(case: str, **ratios) -> None:
@@ -35,10 +40,16 @@ def report_observed(case: str, **ratios) -> None:
 def adv_atol(dtype, seq_len: int) -> float:
     """Advantages of the whole path depend on w_n = exp(sum of up to seq_len token log-probs).
     With float32 logits each row's log-sum-exp carries a few 1e-9 of error (float32 exponentials
-    and differences, averaged over the vocabulary), which adds up over the generation; the
+    and differences, averaged over the vocabulary), with bf16 logits up to 2e-8 where the softmax
+    is very peaked (2e-9 on the benchmark's logits); it adds up over the generation, and the
     advantage inherits it through mean(c R) with c <= eta = 2.  So the bound grows with L."""
-    per_token = 4e-9 if dtype == torch.float32 else 4e-7
+    per_token = 4e-9 if dtype == torch.float32 else 5e-8
     return max(ADV_ATOL[dtype], per_token * seq_len)
+
+
+def head_adv_atol(seq_len: int) -> float:
+    """The same for the fused LM-head form (bf16 operands, float statistics per 256-column tile)."""
+    return max(HEAD_ADV_ATOL, 4e-7 * seq_len)
 
 
 def loss_scale(o) -> float:

@@ -33,7 +33,7 @@ pytestmark = pytest.mark.gpu
 import oracle  # noqa: E402
 from paper_2510_03515_b200 import binding as rb  # noqa: E402
 from paper_2510_03515_b200 import synth  # noqa: E402
-from parity_util import LOGP_ATOL, LOSS_RTOL, adv_atol  # noqa: E402
+from parity_util import HEAD_LOGP_ATOL, LOSS_RTOL, head_adv_atol  # noqa: E402
 
 
 def bf16_to_f64(bits):
@@ -115,10 +115,10 @@ def compare_head(o, g, w):
     dt = torch.bfloat16
     assert g["stats"]["status"] == 0
     slack = o["logp_slack"]
-    assert (np.abs(g["token_logp"] - o["token_logp"]) <= LOGP_ATOL[dt] + slack).all()
-    assert np.median(slack) < 5 * LOGP_ATOL[dt], "the relaxation must stay small against the tolerance itself"
+    assert (np.abs(g["token_logp"] - o["token_logp"]) <= HEAD_LOGP_ATOL + slack).all()
+    assert np.median(slack) < 5 * HEAD_LOGP_ATOL, "the relaxation must stay small against the tolerance itself"
     seq_slack = slack.reshape(w.n_seq, w.seq_len).sum(1).max() * 2.0    # w_n = exp(sum of them), c <= 2
-    np.testing.assert_allclose(g["adv"], o["adv64"], rtol=0, atol=adv_atol(dt, w.seq_len) + seq_slack)
+    np.testing.assert_allclose(g["adv"], o["adv64"], rtol=0, atol=head_adv_atol(w.seq_len) + seq_slack)
     scale = max(abs(o["loss"]), 1e-3 * float(np.abs(o["coef"] * o["seq_logp"]).sum()), 1e-30)
     assert abs(g["loss"] - o["loss"]) / scale <= LOSS_RTOL[dt] + float(np.abs(np.repeat(o["coef"], w.seq_len)) @ slack) / scale
     assert g["stats"]["n_tokens"] == o["stats"]["n_tokens"]
@@ -277,7 +277,7 @@ def _oracle_over_all_rows(w, dev, block):
         g_row = np.repeat(f["coef"], L)
         # relative uncertainty of each generation's coefficient that the advantage tolerance leaves
         seq_slack = f["slack"].reshape(w.n_seq, L).sum(1).max() * 2.0
-        dg = ga["clipped_w"] * (1.0 + np.abs(ga["adv64"])) * (adv_atol(torch.bfloat16, L) + seq_slack) / w.n_seq
+        dg = ga["clipped_w"] * (1.0 + np.abs(ga["adv64"])) * (head_adv_atol(L) + seq_slack) / w.n_seq
         g_rel = np.repeat(np.where(f["coef"] != 0.0, dg / np.maximum(np.abs(f["coef"]), 1e-300), 0.0), L)
         dz = oracle.dlogits_f64_inplace(f["z_rows"].copy(), tg[sel_rows], f["lse"][sel_rows], g_row[sel_rows])
         f["dh_rows"] = oracle.head_dhidden(dz, w_bits)
@@ -329,11 +329,11 @@ def test_fused_head_full_size_config(full_size_oracle, form, flags):
 
     slack = f["slack"]
     lp_err = np.abs(tl.cpu().numpy() - f["lp"])
-    assert (lp_err <= LOGP_ATOL[dt] + slack).all(), f"token log-prob: worst {(lp_err / (LOGP_ATOL[dt] + slack)).max():.2f} x bound"
-    assert np.median(slack) < 5 * LOGP_ATOL[dt]
+    assert (lp_err <= HEAD_LOGP_ATOL + slack).all(), f"token log-prob: worst {(lp_err / (HEAD_LOGP_ATOL + slack)).max():.2f} x bound"
+    assert np.median(slack) < 5 * HEAD_LOGP_ATOL
     seq_slack = slack.reshape(w.n_seq, L).sum(1).max() * 2.0
     adv_err = np.abs(adv.cpu().numpy() - f["adv64"])
-    assert (adv_err <= adv_atol(dt, L) + seq_slack).all()
+    assert (adv_err <= head_adv_atol(L) + seq_slack).all()
     scale = max(abs(f["loss"]), 1e-3 * float(np.abs(f["coef"] * f["seq_logp"]).sum()), 1e-30)
     loss_bound = LOSS_RTOL[dt] + float(np.abs(np.repeat(f["coef"], L)) @ slack) / scale
     loss_rel = abs(loss.item() - f["loss"]) / scale
@@ -358,8 +358,8 @@ def test_fused_head_full_size_config(full_size_oracle, form, flags):
     assert abs(a - c) <= 1e-3 * max(abs(a), abs(c)) + 1e-2, (a, c)
     dead = torch.from_numpy(np.repeat(f["coef"] == 0.0, L)).to(dev)
     assert (dh[dead] == 0).all()
-    report_observed(f"fused head full size ({form} logits)", token_logp=(lp_err / (LOGP_ATOL[dt] + slack)).max(),
-                    adv=(adv_err / (adv_atol(dt, L) + seq_slack)).max(), loss=loss_rel / loss_bound,
+    report_observed(f"fused head full size ({form} logits)", token_logp=(lp_err / (HEAD_LOGP_ATOL + slack)).max(),
+                    adv=(adv_err / (head_adv_atol(L) + seq_slack)).max(), loss=loss_rel / loss_bound,
                     dh=dh_ratio.max(), dW=dW_ratio.max(), loss_rel_abs=loss_rel,
                     coef_term_share_of_dh_bound_at_worst=f["dh_coef_share"].flat[dh_ratio.argmax()])
 
