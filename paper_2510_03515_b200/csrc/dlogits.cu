@@ -8,7 +8,8 @@
 //                     read: one thread per CTA issues bulk shared->global copies from a zeroed
 //                     buffer, which keeps the write stream in large bursts.
 //
-//  dlogits_kernel     live rows.  Persistent CTAs take rows grid-stride.  One producer thread
+//  dlogits_kernel     live rows.  Persistent CTAs draw rows from a counter (the live rows are spread
+//                     unevenly: masked rows cluster at the end of every generation).  One producer thread
 //                     streams each row into a ring of shared-memory stages with bulk global->shared
 //                     copies, running ahead across row boundaries.  Eight consumer warps wait on a
 //                     stage's barrier, turn the logits into dlogits IN PLACE in shared memory, and
@@ -91,7 +92,7 @@ template <int DT>
 __global__ void __launch_bounds__(kThreads)
 dlogits_kernel(const void* logits, void* dlogits /* may alias logits */, int64_t ld, int vocab,
                int seq_len, int64_t row0, int64_t n_rows, const int32_t* __restrict__ targets,
-               rapid_stats_t* stats_user, Workspace ws) {
+               rapid_stats_t* stats_user, unsigned int* ticket /* zero at launch */, Workspace ws) {
     constexpr int ESIZE = (DT == RAPID_BF16) ? 2 : 4;
     constexpr int PER = 16 / ESIZE;  // elements per 16-byte vector
     using RowConst = typename std::conditional<DT == RAPID_BF16, RowConstBf16, RowConstF32>::type;
@@ -100,6 +101,10 @@ dlogits_kernel(const void* logits, void* dlogits /* may alias logits */, int64_t
     __shared__ __align__(8) uint64_t full_bar[kStages];
     __shared__ __align__(8) uint64_t empty_bar[kStages];
     __shared__ int abort_flag;
+    // rows the producer has drawn, in the order it loads them; -1 = no more.  The producer is at most
+    // kStages chunks, hence kStages rows, ahead of the consumers.
+    constexpr int kRowQ = kStages + 1;
+    __shared__ long long row_q[kRowQ];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (tid == 0) {
@@ -123,30 +128,42 @@ dlogits_kernel(const void* logits, void* dlogits /* may alias logits */, int64_t
     if (warp == kConsumerWarps) {
         // ------------------------------- producer -------------------------------------------
         if (lane == 0) {
-            uint32_t it = 0;
+            uint32_t it = 0, j = 0;
             bool ok = true;
-            for (int64_t i = blockIdx.x; i < n_rows && ok; i += gridDim.x) {
-                if (!row_is_live(ws, row0 + i, seq_len)) continue;
+            auto stage_free = [&](uint32_t k) {  // the stage that load k goes into has been given back
+                const uint32_t use = k / kStages;
+                return use == 0 || mbar_wait_bounded(&empty_bar[k % kStages], (use & 1u) ^ 1u, abortp);
+            };
+            while (ok) {
+                int64_t i;
+                do {  // draw rows until a live one comes, or none is left
+                    i = (int64_t)atomicAdd(ticket, 1u);
+                } while (i < n_rows && !row_is_live(ws, row0 + i, seq_len));
+                if (i >= n_rows) break;
                 const uint8_t* src = static_cast<const uint8_t*>(logits) + (size_t)i * ld * ESIZE;
                 for (int c = 0; c < n_chunks; ++c, ++it) {
                     const int s = it % kStages;
-                    const uint32_t use = it / kStages;
-                    if (use > 0 && !mbar_wait_bounded(&empty_bar[s], (use & 1u) ^ 1u, abortp)) {
+                    if (!stage_free(it)) {
                         ok = false;
                         break;
                     }
+                    if (c == 0) row_q[j++ % kRowQ] = i;  // published by the arrive below (release)
                     const int bytes = min(kChunk, load_bytes - c * kChunk);
                     mbar_arrive_expect_tx(&full_bar[s], (uint32_t)bytes);
                     bulk_load(ring + (size_t)s * kChunk, src + (size_t)c * kChunk, (uint32_t)bytes,
                               &full_bar[s]);
                 }
             }
+            if (ok && stage_free(it)) {  // tell the consumers that this was the last row
+                row_q[j % kRowQ] = -1;
+                mbar_arrive(&full_bar[it % kStages]);
+            }
             if (!ok || *abortp) {
                 // gave up: let the copies already issued land before the CTA's memory goes away
                 const uint32_t first = it > (uint32_t)kStages ? it - kStages : 0u;
-                for (uint32_t j = first; j < it; ++j) {
+                for (uint32_t k = first; k < it; ++k) {
                     const unsigned long long t0 = global_timer_ns();
-                    while (!mbar_try_wait(&full_bar[j % kStages], (j / kStages) & 1u))
+                    while (!mbar_try_wait(&full_bar[k % kStages], (k / kStages) & 1u))
                         if (global_timer_ns() - t0 > kWaitLimitNs) break;
                 }
             }
@@ -155,9 +172,14 @@ dlogits_kernel(const void* logits, void* dlogits /* may alias logits */, int64_t
         // ------------------------------- consumers ------------------------------------------
         uint32_t it = 0;
         bool ok = true;
-        for (int64_t i = blockIdx.x; i < n_rows && ok; i += gridDim.x) {
+        for (uint32_t j = 0; ok; ++j) {
+            // the row's first chunk (or the end mark) is what tells which row this is; whether it came is
+            // settled by all consumers together, so that the decision to go on, stop or give up is uniform
+            bool got = mbar_wait_bounded(&full_bar[it % kStages], (it / kStages) & 1u, abortp);
+            if (consumer_barrier_or<kConsumers>(!got || *abortp != 0)) break;
+            const int64_t i = (int64_t)row_q[j % kRowQ];
+            if (i < 0) break;
             const int64_t r = row0 + i;
-            if (!row_is_live(ws, r, seq_len)) continue;
             const int n = (int)(r / seq_len);
             const double g = ws.coef[n];
             uint8_t* orow = static_cast<uint8_t*>(dlogits) + (size_t)i * ld * ESIZE;
@@ -177,7 +199,7 @@ dlogits_kernel(const void* logits, void* dlogits /* may alias logits */, int64_t
                 const int s = it % kStages;
                 // A wait that gives up raises the abort flag; the thread still goes to the barrier
                 // below, which ORs every consumer's view, so all leave together.
-                const bool got = mbar_wait_bounded(&full_bar[s], (it / kStages) & 1u, abortp);
+                if (c > 0) got = mbar_wait_bounded(&full_bar[s], (it / kStages) & 1u, abortp);
                 uint4* sv = reinterpret_cast<uint4*>(ring + (size_t)s * kChunk);
                 const int v0 = c * kVecPerChunk;                  // first vector of the chunk in the row
                 const int nv = min(kVecPerChunk, nvec_row - v0);  // whole real vectors in the chunk
@@ -190,14 +212,14 @@ dlogits_kernel(const void* logits, void* dlogits /* may alias logits */, int64_t
                     }
                     uint4 z[kVecPerThread];
 #pragma unroll
-                    for (int j = 0; j < kVecPerThread; ++j) {
-                        const int v = tid + j * kConsumers;
-                        if (v < nv) z[j] = sv[v];
+                    for (int jj = 0; jj < kVecPerThread; ++jj) {
+                        const int v = tid + jj * kConsumers;
+                        if (v < nv) z[jj] = sv[v];
                     }
 #pragma unroll
-                    for (int j = 0; j < kVecPerThread; ++j) {
-                        const int v = tid + j * kConsumers;
-                        if (v < nv) sv[v] = dz_vec_any(z[j], (v0 + v) * PER, rc);
+                    for (int jj = 0; jj < kVecPerThread; ++jj) {
+                        const int v = tid + jj * kConsumers;
+                        if (v < nv) sv[v] = dz_vec_any(z[jj], (v0 + v) * PER, rc);
                     }
                     fence_proxy_async_smem();  // generic writes above -> asynchronous read below
                 }
@@ -247,8 +269,11 @@ cudaError_t launch_one(const rapid_desc_t& d, const void* logits_chunk, void* dl
     if (per_sm < 1) per_sm = 1;
     int64_t grid = (int64_t)sm_count * per_sm;
     if (grid > n_rows) grid = n_rows;
-    dlogits_kernel<DT><<<(unsigned)grid, kThreads, smem, stream>>>(
-        logits_chunk, dlogits_chunk, d.ld, d.vocab, d.seq_len, row0, n_rows, targets, stats_user, ws);
+    if (n_rows > 0xffffffffll) return cudaErrorInvalidValue;  // the row counter is 32 bits wide
+    e = cudaMemsetAsync(ws.row_ticket, 0, sizeof(unsigned int), stream);
+    if (e != cudaSuccess) return e;
+    dlogits_kernel<DT><<<(unsigned)grid, kThreads, smem, stream>>>(logits_chunk, dlogits_chunk, d.ld, d.vocab, d.seq_len,
+                                                                  row0, n_rows, targets, stats_user, ws.row_ticket, ws);
     return cudaGetLastError();
 }
 

@@ -57,10 +57,13 @@ constexpr int kStages = RAPID_OP_STAGES;
 #endif
 constexpr int kMaxPending = RAPID_OP_PENDING;  // bulk stores that may still be reading their stage
 #ifndef RAPID_OP_RETAIN
-#define RAPID_OP_RETAIN 2
+#define RAPID_OP_RETAIN 0
 #endif
 // The last kRetain chunks of a row's first sweep are not given back to the producer: they stay in their
-// stages, and the second sweep starts on them in place instead of loading them again.
+// stages, and the second sweep starts on them in place instead of loading them again.  Measured slower at
+// every depth (0: 5.79 ms, 1: 5.89, 2: 5.91, 3 with two pending stores: 6.13 on the 64 x 1024 x 151936
+// mini-batch): a stage that is held is a stage the ring cannot load into, and that costs more than the
+// saved loads bring.  Kept as an option, off.
 constexpr int kRetain = RAPID_OP_RETAIN;
 static_assert(kRetain >= 0 && kRetain + kMaxPending < RAPID_OP_STAGES, "retained stages, stages that pending stores hold and one to load into");
 static_assert(kStages >= kMaxPending + 2, "the ring must keep cycling while stores are in flight");
