@@ -333,7 +333,7 @@ template <int DT>
 __global__ void __launch_bounds__(kThreads, RAPID_OP_MINBLOCKS)
 onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, int64_t ld, int vocab, int seq_len,
                      int64_t n_rows, const int32_t* __restrict__ targets, const uint8_t* __restrict__ mask,
-                     int want_logp, Workspace ws) {
+                     int want_logp, unsigned int* ticket /* zero at launch */, unsigned long long stride, Workspace ws) {
     constexpr int ESIZE = (DT == RAPID_BF16) ? 2 : 4;
     constexpr int PER = 16 / ESIZE;
     constexpr bool kBase2 = (DT == RAPID_BF16);
@@ -350,6 +350,10 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
     __shared__ double sh_lse;
     __shared__ float sh_M;
     __shared__ float sh_zy;
+    // rows that are read, in the order the producer loads them: 4 * row + plan; -1 = no more.  The
+    // producer is at most kStages chunks, hence kStages rows, ahead of the consumers.
+    constexpr int kRowQ = kStages + 1;
+    __shared__ long long row_q[kRowQ];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (tid == 0) {
@@ -369,17 +373,12 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
     const int n_chunks = (load_bytes + kChunk - 1) / kChunk;
     const int nvec_row = vocab / PER;
     const int whole = nvec_row * 16;  // bytes of a row in whole vectors of real columns
-    // CTA b owns rows b, b + grid, b + 2 grid, ... and walks them starting at a turn proportional to b,
-    // wrapping around: at any moment the CTAs are spread over the whole batch, so the memory system sees
-    // the batch's average mix of rows that are read and written and rows that are only zero-filled
-    // instead of one kind after the other.
-    const int64_t n_turns = (n_rows + gridDim.x - 1) / gridDim.x;
-    const int64_t turn0 = (n_turns * blockIdx.x) / gridDim.x;
-    auto row_of_turn = [&](int64_t k) -> int64_t {
-        int64_t i = turn0 + k;
-        if (i >= n_turns) i -= n_turns;
-        return i * gridDim.x + blockIdx.x;
-    };
+    // Rows are drawn from a counter, so every CTA stays busy until the rows run out however unevenly the
+    // rows that are read and the rows that are only zero-filled are spread.  Draw t stands for row
+    // (t * stride) mod n_rows, with stride coprime to n_rows and about 0.62 n_rows: rows drawn at about the
+    // same time lie far apart, so the memory system sees the batch's average mix of the two kinds rather
+    // than one kind after the other (masked rows cluster at the end of every generation).
+    auto row_of_draw = [&](unsigned int t) -> int64_t { return (int64_t)(((unsigned long long)t * stride) % (unsigned long long)n_rows); };
 
     if (warp == kConsumerWarps) {
         // ------------------------------- producer -------------------------------------------
@@ -387,18 +386,33 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
             const uint64_t keep = policy_evict_last(), stream = policy_evict_first();
             uint32_t it = 0;
             bool ok = true;
-            for (int64_t k = 0; k < n_turns && ok; ++k) {
-                const int64_t r = row_of_turn(k);
-                if (r >= n_rows) continue;
+            uint32_t jq = 0;
+            auto stage_free = [&](uint32_t k) {  // the stage that load k goes into has been given back
+                const uint32_t use = k / kStages;
+                return use == 0 || mbar_wait_bounded(&empty_bar[k % kStages], (use & 1u) ^ 1u, abortp);
+            };
+            while (ok) {
+                const unsigned int t = atomicAdd(ticket, 1u);
+                if ((int64_t)t >= n_rows) break;
+                const int64_t r = row_of_draw(t);
                 uint8_t st;
                 const int plan = row_plan(r, seq_len, vocab, targets, mask, ws, want_logp != 0, &st);
                 if (plan == ROWS_NONE) {
-                    // a row nobody reads gets its zeros from here, ahead of the consumers and outside their
-                    // accounting of pending stores (whole vectors; the consumers write the few columns after them)
+                    // a row nobody reads is finished here: zeros from the zero buffer (whole vectors by bulk
+                    // copies, outside the consumers' accounting of pending stores; the few columns after them
+                    // one by one) and its entries of the per-row statistics
                     uint8_t* orow = static_cast<uint8_t*>(dlogits) + (size_t)r * ld * ESIZE;
                     for (int o = 0; o < whole; o += kZeroBuf)
                         bulk_store_hint(orow + o, zeros, (uint32_t)min(kZeroBuf, whole - o), stream);
                     bulk_commit();
+                    for (int e = nvec_row * PER; e < vocab; ++e) {
+                        if (ESIZE == 2) reinterpret_cast<uint16_t*>(orow)[e] = 0;
+                        else reinterpret_cast<float*>(orow)[e] = 0.f;
+                    }
+                    ws.row_state[r] = st;
+                    ws.lse[r] = 0.0;
+                    ws.token_logp[r] = 0.0;
+                    ws.row_max[r] = 0.f;
                     continue;
                 }
                 const uint8_t* src = static_cast<const uint8_t*>(logits) + (size_t)r * ld * ESIZE;
@@ -409,17 +423,21 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
                     const int n_load = (sweep == 1) ? n_chunks - min(kRetain, n_chunks) : n_chunks;
                     for (int c = 0; c < n_load; ++c, ++it) {
                         const int s = it % kStages;
-                        const uint32_t use = it / kStages;
-                        if (use > 0 && !mbar_wait_bounded(&empty_bar[s], (use & 1u) ^ 1u, abortp)) {
+                        if (!stage_free(it)) {
                             ok = false;
                             break;
                         }
+                        if (sweep == 0 && c == 0) row_q[jq++ % kRowQ] = 4 * r + plan;  // published by the arrive below
                         const int bytes = min(kChunk, load_bytes - c * kChunk);
                         mbar_arrive_expect_tx(&full_bar[s], (uint32_t)bytes);
                         bulk_load_hint(ring + (size_t)s * kChunk, src + (size_t)c * kChunk, (uint32_t)bytes,
                                        &full_bar[s], pol);
                     }
                 }
+            }
+            if (ok && stage_free(it)) {  // tell the consumers that this was the last row
+                row_q[jq % kRowQ] = -1;
+                mbar_arrive(&full_bar[it % kStages]);
             }
             if (!ok || *abortp) {
                 const uint32_t first = it > (uint32_t)kStages ? it - kStages : 0u;
@@ -482,13 +500,16 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
         };
         static_assert(kMaxPending >= 1 && kMaxPending <= 6, "drain_one covers up to six pending stores");
 
-        // After a timeout a warp stops working (ok = false) but keeps walking the rows, so that it
-        // still meets the others at the next live row's barrier, where all agree to leave.
-        for (int64_t k = 0; k < n_turns; ++k) {
-            const int64_t r = row_of_turn(k);
-            if (r >= n_rows) continue;
-            uint8_t state;
-            const int plan = row_plan(r, seq_len, vocab, targets, mask, ws, want_logp != 0, &state);
+        // A row starts when its first chunk has landed; the queue entry published with it says which row
+        // it is.  Whether it came is settled by all consumers together: after a timeout a warp stops
+        // working (ok = false) but still comes here, where all agree to leave.
+        for (uint32_t jq = 0;; ++jq) {
+            const bool came = ok && mbar_wait_bounded(&full_bar[st], ph, abortp);
+            if (consumer_barrier_or<kConsumers>(!came || *abortp != 0)) break;
+            const long long entry = row_q[jq % kRowQ];
+            if (entry < 0) break;
+            const int64_t r = entry >> 2;
+            const int plan = (int)(entry & 3);
             uint8_t* orow = static_cast<uint8_t*>(dlogits) + (size_t)r * ld * ESIZE;
             // rows without gradient get zeros, straight from the zero buffer (after the row has been
             // read, if it is read at all: dlogits may be the logits buffer itself)
@@ -503,19 +524,6 @@ onpolicy_rows_kernel(const void* logits, void* dlogits /* may alias logits */, i
                     else reinterpret_cast<float*>(orow)[nvec_row * PER + tid - 1] = 0.f;
                 }
             };
-            if (plan == ROWS_NONE) {  // the producer sends the zeros
-                if (nvec_row * PER + tid < vocab) {
-                    if (ESIZE == 2) reinterpret_cast<uint16_t*>(orow)[nvec_row * PER + tid] = 0;
-                    else reinterpret_cast<float*>(orow)[nvec_row * PER + tid] = 0.f;
-                }
-                if (tid == 0) {
-                    ws.row_state[r] = state;
-                    ws.lse[r] = 0.0;
-                    ws.token_logp[r] = 0.0;
-                    ws.row_max[r] = 0.f;
-                }
-                continue;
-            }
             const int y = targets[r];
             // ---- sweep 1: max and sum of exponentials.  Each warp owns a contiguous slice of every
             // chunk and gives the stage back on its own (the stage's barrier counts the warps), so no
@@ -751,6 +759,22 @@ onpolicy_loss_kernel(int n_seq, float* __restrict__ loss_out, rapid_stats_t* __r
 
 }  // namespace
 
+// A multiplier coprime to n and near 0.62 n: t -> (t * stride) mod n visits every row once, neighbours in t far apart.
+static unsigned long long scatter_stride(int64_t n) {
+    auto gcd = [](unsigned long long a, unsigned long long b) {
+        while (b) {
+            const unsigned long long c = a % b;
+            a = b;
+            b = c;
+        }
+        return a;
+    };
+    unsigned long long s = (unsigned long long)((double)n * 0.6180339887498949);
+    if (s < 1) s = 1;
+    while (gcd(s, (unsigned long long)n) != 1) ++s;
+    return s;
+}
+
 cudaError_t launch_onpolicy(const rapid_desc_t& d, const void* logits, void* dlogits, const int32_t* targets,
                             const uint8_t* mask, const float* rewards, const int32_t* group_offsets, float* loss,
                             float* token_logp, float* adv, rapid_stats_t* stats, const Workspace& ws, int sm_count,
@@ -771,8 +795,11 @@ cudaError_t launch_onpolicy(const rapid_desc_t& d, const void* logits, void* dlo
         if (per_sm < 1) per_sm = 1;
         int64_t grid = (int64_t)sm_count * per_sm;
         if (grid > T) grid = T;
+        if (T > 0xffffffffll) return cudaErrorInvalidValue;  // the row counter is 32 bits wide
+        err = cudaMemsetAsync(ws.row_ticket, 0, sizeof(unsigned int), stream);
+        if (err != cudaSuccess) return err;
         kern<<<(unsigned)grid, kThreads, smem, stream>>>(logits, dlogits, d.ld, d.vocab, d.seq_len, T, targets, mask,
-                                                         want_logp, ws);
+                                                         want_logp, ws.row_ticket, scatter_stride(T), ws);
         return cudaGetLastError();
     };
     e = (d.dtype == RAPID_BF16) ? go(onpolicy_rows_kernel<RAPID_BF16>) : go(onpolicy_rows_kernel<RAPID_F32>);
