@@ -341,14 +341,14 @@ def mean_median(xs):
 # DRAM traffic per algorithmic byte, from the ncu captures summarised under profiles/ (counters
 # dram__bytes_read.sum + dram__bytes_write.sum of a smaller launch of the same kernel; traffic grows
 # in proportion to the rows processed).  NOT counters of this run: the line says so.
-TRAFFIC_P2_PER_BYTE = 0.9715
+TRAFFIC_P2_PER_BYTE = 0.9719
 TRAFFIC_P2_SOURCE = "profiles/logits_in_path_slm_bf16.md: ncu dram bytes of a 2.5 GB launch x rows of this one"
 # the on-policy kernel: dram__bytes_read.sum per byte of live rows, dram__bytes_write.sum per byte of all rows
-TRAFFIC_OP_READ_PER_LIVE_BYTE = 1.285
-TRAFFIC_OP_WRITE_PER_ROW_BYTE = 0.976
+TRAFFIC_OP_READ_PER_LIVE_BYTE = 1.288
+TRAFFIC_OP_WRITE_PER_ROW_BYTE = 0.977
 TRAFFIC_OP_SOURCE = "profiles/onpolicy_rows_kernel_slm_bf16.md: ncu dram bytes of an 8192-row launch x rows of this one"
 # pass 1's secondary ceiling: share of cycles the MUFU (ex2) pipe is busy, same captures
-MUFU_PIPE_PCT_PASS1 = 70.0
+MUFU_PIPE_PCT_PASS1 = 80.2
 MUFU_SOURCE = "profiles/logits_in_path_slm_bf16.md (ncu pipe utilisation of row_stats_kernel)"
 
 
