@@ -588,7 +588,9 @@ def run_fused(args, rk: Rank):
     T, V, D, N = w.n_rows, w.vocab, w.hidden, w.n_seq
     stored = args.head == "stored"
     desc = rb.make_desc(N, w.seq_len, V, w.n_prompts, torch.bfloat16, V, 2.0,
-                        rb.FLAG_HEAD_STORE_LOGITS if stored else 0)
+                        (rb.FLAG_HEAD_STORE_LOGITS if stored else 0) |
+                        (rb.FLAG_HEAD_CTA_PAIRS if getattr(args, "cta_pairs", False) else 0) |
+                        (rb.FLAG_HEAD_SINGLE_CTA if getattr(args, "single_cta", False) else 0))
     ws = rb.alloc_fused_head_workspace(desc, D, dev)
     loss = torch.zeros(1, device=dev)
     dh = torch.empty((T, D), dtype=torch.bfloat16, device=dev)
@@ -669,7 +671,8 @@ def run_fused(args, rk: Rank):
         "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "ms_per_step_median": ms_median,
-        "config": {"workload": "fused", "head": args.head, "prompts": w.n_prompts, "generations_per_prompt": w.group_size,
+        "config": {"workload": "fused", "head": args.head, "ctas_per_tile": ("pairs" if getattr(args, "cta_pairs", False) else "single" if getattr(args, "single_cta", False)
+                                             else "pairs for forward and recompute, single for dhidden and dW"), "prompts": w.n_prompts, "generations_per_prompt": w.group_size,
                    "padded_len": w.seq_len, "rows_per_gpu": T, "hidden": D, "vocab": V,
                    "l2_policy": "inputs larger than L2 (0.47 GB weight, 5 GB dlogits scratch per step)",
                    "eta": 2.0, "parallelism": f"dp{world} (by prompt group, no data-path collective)"},
@@ -840,6 +843,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="slm", choices=["slm", "fused", "onpolicy", "long"],
                     help="slm: the logits-in path the metric is quoted on (default); long: the 64 x 4096 x 32000 fp32 configuration through the chunked form; onpolicy: single pass; fused: the LM-head form")
+    ap.add_argument("--cta-pairs", action="store_true",
+                    help="--workload fused: all four contractions on pairs of CTAs (256 x 256 tiles, tcgen05 cta_group::2)")
+    ap.add_argument("--single-cta", action="store_true",
+                    help="--workload fused: all four contractions on one CTA per 128 x 256 tile (default: the measured-best mix)")
     ap.add_argument("--head", default="recompute", choices=["recompute", "stored"],
                     help="--workload fused: form the logits twice on the tensor cores (four contractions), or keep "
                          "them in bf16 between forward and backward (three contractions)")

@@ -89,7 +89,16 @@ enum {
     /* forming them a second time on the tensor cores: three GEMM-sized contractions instead of    */
     /* four, for one more write and read of [T, vocab] bf16.  The row statistics are then those of */
     /* the rounded logits, i.e. the results are those of rapid_pg_loss_fwd_bwd on bf16(h W).       */
-    RAPID_FLAG_HEAD_STORE_LOGITS = 64u
+    RAPID_FLAG_HEAD_STORE_LOGITS = 64u,
+    /* rapid_pg_loss_fused_head only.  Its contractions run either on one CTA per 128 x 256 tile or  */
+    /* on PAIRS of CTAs (two SMs share one 256 x 256 tile, each holding half of either operand;      */
+    /* tcgen05 cta_group::2; every pair is a thread-block cluster on this GPU alone): same results   */
+    /* to rounding order, a third less operand traffic into shared memory per flop, more power.  By  */
+    /* default the forward and the recompute contraction (K = hidden size) run on pairs and the two  */
+    /* long-K ones (dhidden, dW) on single CTAs, the mix measured fastest; these two flags force     */
+    /* all four one way (CTA_PAIRS wins if both are given).                                          */
+    RAPID_FLAG_HEAD_CTA_PAIRS = 128u,
+    RAPID_FLAG_HEAD_SINGLE_CTA = 256u
 };
 
 /* Problem descriptor (host memory, plain data, 48 bytes). */

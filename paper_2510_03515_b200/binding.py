@@ -35,6 +35,8 @@ FLAG_LEAVE_ONE_OUT = 8
 FLAG_LOO_LITERAL_DIVISOR = 16
 FLAG_NORM_GIVEN = 32
 FLAG_HEAD_STORE_LOGITS = 64
+FLAG_HEAD_CTA_PAIRS = 128
+FLAG_HEAD_SINGLE_CTA = 256
 
 # every symbol declared in include/rapid_pg.h
 EXPORTS = (

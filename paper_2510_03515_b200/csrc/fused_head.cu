@@ -16,6 +16,7 @@
 
 #include "rapid_common.cuh"
 #include "umma_gemm.cuh"
+#include "umma_gemm_pair.cuh"
 
 namespace rapid {
 
@@ -505,6 +506,18 @@ extern "C" rapid_status_t rapid_pg_loss_fused_head(
 
     const int nV = (V + BN - 1) / BN;
     clear_status_kernel<<<1, 1, 0, st>>>(hs.status);
+    // one CTA per 128 x 256 tile, or a pair of CTAs per 256 x 256 tile
+    // Which contractions run on pairs of CTAs (one 256 x 256 tile per two SMs) rather than one CTA per
+    // 128 x 256 tile: bit 0 forward, 1 recompute, 2 dhidden, 3 dW.  Unless a flag says otherwise the two
+    // whose K loop is the hidden size (short, with a heavy epilogue) go to pairs and the two with long K
+    // loops stay on single CTAs: measured best on the 16384 x 1536 x 151936 configuration at the power cap
+    // (23.45 ms against 24.08 all single and 24.9 all pairs on the same box; pairs need less operand traffic
+    // per flop but draw more power, and the long step settles at a lower clock).
+    const uint32_t pair_mask = (desc->flags & RAPID_FLAG_HEAD_CTA_PAIRS) ? 15u
+                               : (desc->flags & RAPID_FLAG_HEAD_SINGLE_CTA) ? 0u : 3u;
+    const bool pairs = (pair_mask & 4u) != 0;
+    CUtensorMap w_k_half;  // B of dh for a CTA of a pair: 128 of the tile's 256 rows of W^T per box
+    if (pairs && !make_map_bf16(&w_k_half, w_vocab, D, V, ld, BK, BN / 2)) return RAPID_ERR_CUDA;
 
     // forward
     const bool store_z = (desc->flags & RAPID_FLAG_HEAD_STORE_LOGITS) != 0;
@@ -519,11 +532,13 @@ extern "C" rapid_status_t rapid_pg_loss_fused_head(
             fp.targets = targets;
             fp.T = (int)T;
             fp.V = V;
-            if (launch_gemm<FwdStatsStore, false, true>(h_k, w_mn, fwd, sms, hs.status, fp, st) != cudaSuccess)
+            if (((pair_mask & 1u) ? launch_gemm_pair<FwdStatsStore, false, true>(h_k, w_mn, fwd, sms, hs.status, fp, st)
+                       : launch_gemm<FwdStatsStore, false, true>(h_k, w_mn, fwd, sms, hs.status, fp, st)) != cudaSuccess)
                 return RAPID_ERR_CUDA;
         } else {
             FwdStats::Params fp{hs.part_m, hs.part_s, hs.zy, targets, (int)T, V};
-            if (launch_gemm<FwdStats, false, true>(h_k, w_mn, fwd, sms, hs.status, fp, st) != cudaSuccess)
+            if (((pair_mask & 1u) ? launch_gemm_pair<FwdStats, false, true>(h_k, w_mn, fwd, sms, hs.status, fp, st)
+                       : launch_gemm<FwdStats, false, true>(h_k, w_mn, fwd, sms, hs.status, fp, st)) != cudaSuccess)
                 return RAPID_ERR_CUDA;
         }
     }
@@ -570,18 +585,21 @@ extern "C" rapid_status_t rapid_pg_loss_fused_head(
         dzp.seq_len = desc->seq_len;
         dzp.row0 = (int)r0;
         Shape sdz{mR, nV, (D + BK - 1) / BK, M_FASTEST};
-        if (!store_z && launch_gemm<DzStore, false, true>(hc_k, w_mn, sdz, sms, hs.status, dzp, st) != cudaSuccess)
+        if (!store_z && ((pair_mask & 2u) ? launch_gemm_pair<DzStore, false, true>(hc_k, w_mn, sdz, sms, hs.status, dzp, st)
+                               : launch_gemm<DzStore, false, true>(hc_k, w_mn, sdz, sms, hs.status, dzp, st)) != cudaSuccess)
             return RAPID_ERR_CUDA;
 
         dhp.N = D;
         Shape sdh{mR, (D + BN - 1) / BN, (V + BK - 1) / BK, N_FASTEST};
-        if (launch_gemm<StoreBf16, false, false>(dz_k, w_k, sdh, sms, hs.status, dhp, st) != cudaSuccess)
+        if (((pair_mask & 4u) ? launch_gemm_pair<StoreBf16, false, false>(dz_k, w_k_half, sdh, sms, hs.status, dhp, st)
+                   : launch_gemm<StoreBf16, false, false>(dz_k, w_k, sdh, sms, hs.status, dhp, st)) != cudaSuccess)
             return RAPID_ERR_CUDA;
 
         dwp.N = V;
         dwp.accumulate = (r0 > 0) ? 1 : 0;
         Shape sdw{(D + BM - 1) / BM, nV, (int)((R + BK - 1) / BK), M_FASTEST};
-        if (launch_gemm<StoreF32, true, true>(hc_mn, dz_mn, sdw, sms, hs.status, dwp, st) != cudaSuccess)
+        if (((pair_mask & 8u) ? launch_gemm_pair<StoreF32, true, true>(hc_mn, dz_mn, sdw, sms, hs.status, dwp, st)
+                   : launch_gemm<StoreF32, true, true>(hc_mn, dz_mn, sdw, sms, hs.status, dwp, st)) != cudaSuccess)
             return RAPID_ERR_CUDA;
     }
 

@@ -139,17 +139,20 @@ def compare_head(o, g, w):
     assert np.abs(o["dh"]).max() > 100 * tol_h.mean() or np.abs(o["dh"]).max() > 1e-4
 
 
+@pytest.mark.parametrize("extra", [0, rb.FLAG_HEAD_SINGLE_CTA])
 @pytest.mark.parametrize("V,D,L,pad", [(1000, 192, 40, 0), (777, 200, 50, 7), (256, 64, 32, 0), (5000, 1536, 33, 8)])
-def test_fused_head_scaled(V, D, L, pad):
+def test_fused_head_scaled(V, D, L, pad, extra):
     """Ragged everything: rows not a multiple of 128, vocabulary not a multiple of 256 (or of 8),
-    hidden size not a multiple of 64, ragged generation lengths, a padded weight pitch."""
+    hidden size not a multiple of 64, ragged generation lengths, a padded weight pitch.  Once with
+    the default mix of kernels (forward and recompute on CTA pairs, dhidden and dW on single CTAs) and
+    once with every contraction on single CTAs."""
     pad = (-V) % 8 + pad if (V + pad) % 8 else pad
     w = synth.CONFIGS["fused"].scaled(n_prompts=3, group_size=4, seq_len=L, vocab=V, hidden=D,
                                       length_mode="uniform", len_lo=L // 3, reward_mode="per_prompt_const",
                                       seed=300 + V)
     b = synth.make_head(w)
     o = oracle_head(b, w)
-    g = run_head(b, w, o["behav"], ld_pad=pad)
+    g = run_head(b, w, o["behav"], ld_pad=pad, flags=extra)
     compare_head(o, g, w)
     assert np.all(o["adv64"][:4] == 0.0)   # the all-zero-reward group: its rows give no gradient
 
@@ -190,6 +193,39 @@ def test_fused_head_mid_size_many_tiles_per_cta():
     o = oracle_head(b, w)
     g = run_head(b, w, o["behav"])
     compare_head(o, g, w)
+
+
+@pytest.mark.parametrize("V,D,L,pad,extra", [(1000, 192, 40, 0, 0), (777, 200, 50, 7, 0), (5000, 1536, 33, 8, 0),
+                                             (40, 8, 3, 0, 0), (1000, 192, 40, 0, rb.FLAG_HEAD_STORE_LOGITS),
+                                             (5000, 1536, 33, 8, rb.FLAG_HEAD_STORE_LOGITS)])
+def test_fused_head_cta_pairs(V, D, L, pad, extra):
+    """RAPID_FLAG_HEAD_CTA_PAIRS: every contraction on pairs of CTAs (256 x 256 tiles, tcgen05 cta_group::2).
+    Ragged rows (not a multiple of 256, so the second CTA of the last pair is partly or wholly past the
+    end), vocabulary and hidden size; both forms of the head; everything against the dense oracle."""
+    pad = (-V) % 8 + pad if (V + pad) % 8 else pad
+    w = synth.CONFIGS["fused"].scaled(n_prompts=3, group_size=4, seq_len=L, vocab=V, hidden=D,
+                                      length_mode="uniform", len_lo=max(1, L // 3), reward_mode="per_prompt_const",
+                                      seed=300 + V)
+    b = synth.make_head(w)
+    o = oracle_head(b, w, flags=extra)
+    g = run_head(b, w, o["behav"], ld_pad=pad, flags=extra | rb.FLAG_HEAD_CTA_PAIRS)
+    compare_head(o, g, w)
+
+
+def test_fused_head_cta_pairs_many_tiles_and_two_backward_chunks():
+    """Pairs of CTAs over many tiles per pair (2048 x 32000 x 512) and over two backward chunks (18000
+    rows, the second one ragged, its contribution added to dW)."""
+    w = synth.CONFIGS["fused"].scaled(n_prompts=2, group_size=4, seq_len=256, vocab=32000, hidden=512,
+                                      length_mode="uniform", len_lo=100, reward_mode="per_prompt", seed=31)
+    b = synth.make_head(w)
+    o = oracle_head(b, w)
+    compare_head(o, run_head(b, w, o["behav"], flags=rb.FLAG_HEAD_CTA_PAIRS), w)
+    w = synth.CONFIGS["fused"].scaled(n_prompts=3, group_size=3, seq_len=2000, vocab=600, hidden=64,
+                                      length_mode="uniform", len_lo=1500, reward_mode="per_prompt", seed=71)
+    b = synth.make_head(w)
+    b["rewards"] = torch.randn(w.n_seq, generator=torch.Generator().manual_seed(8))
+    o = oracle_head(b, w)
+    compare_head(o, run_head(b, w, o["behav"], flags=rb.FLAG_HEAD_CTA_PAIRS), w)
 
 
 @pytest.fixture(scope="module")
@@ -297,7 +333,9 @@ def _oracle_over_all_rows(w, dev, block):
     return {"w": w, "b": b, "forms": forms, "sel_rows": sel_rows, "cols": cols}
 
 
-@pytest.mark.parametrize("form,flags", [("exact", 0), ("bf16", rb.FLAG_HEAD_STORE_LOGITS)])
+@pytest.mark.parametrize("form,flags", [("exact", 0), ("bf16", rb.FLAG_HEAD_STORE_LOGITS),
+                                        ("exact", rb.FLAG_HEAD_CTA_PAIRS), ("exact", rb.FLAG_HEAD_SINGLE_CTA),
+                                        ("bf16", rb.FLAG_HEAD_STORE_LOGITS | rb.FLAG_HEAD_SINGLE_CTA)])
 def test_fused_head_full_size_config(full_size_oracle, form, flags):
     """The full benchmark configuration against the oracle on every row: all 16 384 token
     log-probabilities, all 64 advantages, the loss, the statistics; dhidden on 48 sampled rows
@@ -358,7 +396,7 @@ def test_fused_head_full_size_config(full_size_oracle, form, flags):
     assert abs(a - c) <= 1e-3 * max(abs(a), abs(c)) + 1e-2, (a, c)
     dead = torch.from_numpy(np.repeat(f["coef"] == 0.0, L)).to(dev)
     assert (dh[dead] == 0).all()
-    report_observed(f"fused head full size ({form} logits)", token_logp=(lp_err / (HEAD_LOGP_ATOL + slack)).max(),
+    report_observed(f"fused head full size ({form} logits{', CTA pairs' if flags & rb.FLAG_HEAD_CTA_PAIRS else ', single CTAs' if flags & rb.FLAG_HEAD_SINGLE_CTA else ''})", token_logp=(lp_err / (HEAD_LOGP_ATOL + slack)).max(),
                     adv=(adv_err / (head_adv_atol(L) + seq_slack)).max(), loss=loss_rel / loss_bound,
                     dh=dh_ratio.max(), dW=dW_ratio.max(), loss_rel_abs=loss_rel,
                     coef_term_share_of_dh_bound_at_worst=f["dh_coef_share"].flat[dh_ratio.argmax()])
