@@ -258,6 +258,16 @@ def free_port() -> int:
         return sk.getsockname()[1]
 
 
+def reduce_over_ranks(dist, device, x: float, op: str) -> float:
+    """MAX or SUM of one number over the ranks of `dist` (the only things that ever cross ranks here:
+    the timed interval and the token count); the number itself when there is one rank."""
+    if dist is None:
+        return float(x)
+    t = torch.tensor([x], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX if op == "max" else dist.ReduceOp.SUM)
+    return float(t.item())
+
+
 class Rank:
     """This process's place among the ranks; the NCCL group carries only timings and token counts."""
 
@@ -284,18 +294,10 @@ class Rank:
             self.dist.barrier()
 
     def max_over_ranks(self, x: float) -> float:
-        if not self.dist:
-            return float(x)
-        t = torch.tensor([x], device=self.dev, dtype=torch.float64)
-        self.dist.all_reduce(t, op=self.dist.ReduceOp.MAX)
-        return float(t.item())
+        return reduce_over_ranks(self.dist, self.dev, x, "max")
 
     def sum_over_ranks(self, x: float) -> float:
-        if not self.dist:
-            return float(x)
-        t = torch.tensor([x], device=self.dev, dtype=torch.float64)
-        self.dist.all_reduce(t, op=self.dist.ReduceOp.SUM)
-        return float(t.item())
+        return reduce_over_ranks(self.dist, self.dev, x, "sum")
 
     def close(self):
         if self.dist and self.dist.is_initialized():
@@ -769,6 +771,11 @@ def run_onpolicy(args, rk: Rank):
         return None
     ms_per_step = ms / args.steps
     st = rb.read_stats(stats)
+    cpu = None
+    if not args.skip_cpu:   # the oracle's steps 1-6 on a bounded sample of the same mini-batch shape
+        cpu = oracle_sample(w, target_seconds=args.cpu_seconds, single_thread=False)
+        for k in ("seconds", "tokens", "single_thread"):
+            cpu.pop(k, None)
     peak, peak_kind = load_peaks()
     row_bytes = V * (2 if w.dtype == "bf16" else 4)
     algo = live_rows * 2 * row_bytes + (T - live_rows) * row_bytes   # live rows: one read + one write
@@ -790,7 +797,7 @@ def run_onpolicy(args, rk: Rank):
                      "peak_kind": peak_kind, "unit": "GB/s", "frac": ach / peak, "frac_of_8TBs_nominal": ach / 8000.0,
                      "achieved_at_median": algo / (ms_median * 1e-3) / 1e9,
                      "algorithmic_bytes_per_launch": algo, "traffic": traffic, "traffic_source": TRAFFIC_OP_SOURCE},
-        "cpu_baseline": None, "stats": {"loss": st["loss"], "status": st["status"]},
+        "cpu_baseline": cpu, "stats": {"loss": st["loss"], "status": st["status"]},
     }
     return line
 

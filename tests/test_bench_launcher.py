@@ -37,3 +37,33 @@ def test_inside_a_launcher_the_rank_count_must_match():
 def test_free_port_is_usable():
     p = bench.free_port()
     assert 1024 < p < 65536
+
+
+def _rank_worker(rank, world, port, out):
+    import torch.distributed as dist
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        # what a rank contributes: its own timed interval and its own token count
+        ms = bench.reduce_over_ranks(dist, "cpu", 7.0 + rank, "max")
+        tokens = bench.reduce_over_ranks(dist, "cpu", 1000.0 * (rank + 1), "sum")
+        out.put((rank, ms, tokens))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_timing_is_the_maximum_and_tokens_the_sum_over_ranks():
+    """Two ranks (gloo, CPU): the step time of the job is the slowest rank's, the tokens are everyone's."""
+    import torch.multiprocessing as mp
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = bench.free_port()
+    procs = [ctx.Process(target=_rank_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = sorted(out.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert got == [(0, 8.0, 3000.0), (1, 8.0, 3000.0)]
+    assert bench.reduce_over_ranks(None, "cpu", 5.5, "max") == 5.5
