@@ -452,7 +452,7 @@ def run_ours(args, rk: Rank):
         "clocks": clocks,
         "e2e": e2e,
         "e2e_gradient_to_host": e2e_grad,
-        "gpu_launches": (2 + 3 * n_chunks) * args.steps,
+        "gpu_launches": (2 + 2 * n_chunks) * args.steps,
         "roofline": {"bound": "hbm", "kernel": "dlogits_kernel (pass 2)", "achieved": ach_p2,
                      "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": ach_p2 / peak,
                      "frac_of_8TBs_nominal": ach_p2 / 8000.0, "ms_per_launch": p2 / n_chunks,
@@ -678,7 +678,7 @@ def run_fused(args, rk: Rank):
                    "padded_len": w.seq_len, "rows_per_gpu": T, "hidden": D, "vocab": V,
                    "l2_policy": "inputs larger than L2 (0.47 GB weight, 5 GB dlogits scratch per step)",
                    "eta": 2.0, "parallelism": f"dp{world} (by prompt group, no data-path collective)"},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": (10 if stored else 9) * args.steps,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": 9 * args.steps,
         "roofline": {"bound": "tensor",
                      "kernel": ("umma gemm_kernel x3 (forward statistics + logits store, dhidden, dW); dlogits in place "
                                 "by the logits-in second pass") if stored else

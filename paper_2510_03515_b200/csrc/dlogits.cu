@@ -2,22 +2,24 @@
 //     dlogits[r, v] = g_n m_r (softmax(z[r, .])_v - 1[v == y_r]),
 // the derivative of the Eq. 3 surrogate loss through the log-softmax.
 //
-// Two kernels, both HBM-bound:
+// One kernel, HBM-bound.  Persistent CTAs draw rows from a counter, scattered over the block of rows
+// (draw t stands for row (t * stride) mod rows, stride coprime to the row count), because the two kinds
+// of rows are spread unevenly: masked rows cluster at the end of every generation.
 //
-//  zero_rows_kernel   rows that are masked, or whose coefficient g_n is zero, get zeros.  Nothing is
-//                     read: one thread per CTA issues bulk shared->global copies from a zeroed
-//                     buffer, which keeps the write stream in large bursts.
+//  rows that are masked, or whose coefficient g_n is zero, get zeros and nothing is read: each CTA's
+//  producer thread sends them straight from a zeroed shared-memory buffer with bulk shared->global
+//  copies -- all of them before it starts on the live rows when the launch is large, between the
+//  loads of the live rows when it is small.
 //
-//  dlogits_kernel     live rows.  Persistent CTAs draw rows from a counter (the live rows are spread
-//                     unevenly: masked rows cluster at the end of every generation).  One producer thread
-//                     streams each row into a ring of shared-memory stages with bulk global->shared
-//                     copies, running ahead across row boundaries.  Eight consumer warps wait on a
-//                     stage's barrier, turn the logits into dlogits IN PLACE in shared memory, and
-//                     one of them sends the stage back out with a bulk shared->global copy; the
-//                     stage returns to the producer once that copy has finished reading it.  Bytes
-//                     in flight are set by the ring, not by registers, and both directions move in
-//                     bursts of kChunk bytes.  A chunk is fully read before any of it is
-//                     overwritten, so dlogits may be the logits buffer itself.
+//  live rows: the producer thread draws rows from the first counter, passes over the dead ones, streams
+//  each live row into a ring of shared-memory stages with bulk
+//  global->shared copies, running ahead across row boundaries, and publishes the row's number
+//  through a small queue.  Eight consumer warps wait on a stage's barrier, turn the logits into
+//  dlogits IN PLACE in shared memory, and one of them sends the stage back out with a bulk
+//  shared->global copy; the stage returns to the producer once that copy has finished reading it.
+//  Bytes in flight are set by the ring, not by registers, and both directions move in bursts of
+//  kChunk bytes.  A chunk is fully read before any of it is overwritten, so dlogits may be the
+//  logits buffer itself.
 //
 // The arithmetic of one vector of a row is in dz_rows.cuh (shared with the on-policy kernel).
 #include "dz_rows.cuh"
@@ -50,54 +52,26 @@ constexpr int kVecPerThread = kVecPerChunk / kConsumers;
 static_assert(kVecPerChunk % kConsumers == 0, "chunk must be a multiple of 16 B x consumers");
 static_assert(kStages >= 3, "need a stage to load, one to work on and one to store");
 
-constexpr int kZeroThreads = 128;
-constexpr int kZeroBuf = 16384;
+constexpr int kZeroBuf = 8192;  // zeroed shared memory that the fills of rows without gradient are sent from
 
 __device__ __forceinline__ bool row_is_live(const Workspace& ws, int64_t r, int seq_len) {
     return ws.row_state[r] == ROW_OK && ws.coef[(int)(r / seq_len)] != 0.0;
 }
 
-// ---- dead rows ------------------------------------------------------------------------------------
-
-template <int ESIZE>
-__global__ void __launch_bounds__(kZeroThreads)
-zero_rows_kernel(void* dlogits, int64_t ld, int vocab, int seq_len, int64_t row0, int64_t n_rows,
-                 Workspace ws) {
-    __shared__ __align__(128) uint8_t zeros[kZeroBuf];
-    const int tid = threadIdx.x;
-    for (int i = tid; i < kZeroBuf / 16; i += kZeroThreads)
-        reinterpret_cast<uint4*>(zeros)[i] = make_uint4(0, 0, 0, 0);
-    fence_proxy_async_smem();
-    __syncthreads();
-    const int whole = (vocab * ESIZE) / 16 * 16;  // bytes of a row in whole 16-byte vectors
-    const int tail0 = whole / ESIZE;              // first column not covered by them
-    for (int64_t i = blockIdx.x; i < n_rows; i += gridDim.x) {
-        const int64_t r = row0 + i;
-        if (row_is_live(ws, r, seq_len)) continue;
-        uint8_t* orow = static_cast<uint8_t*>(dlogits) + (size_t)i * ld * ESIZE;
-        if (tid == 0) {
-            for (int o = 0; o < whole; o += kZeroBuf) bulk_store(orow + o, zeros, (uint32_t)min(kZeroBuf, whole - o));
-            bulk_commit();
-        } else if (tail0 + (tid - 1) < vocab) {  // fewer than 16 bytes of ragged tail
-            if (ESIZE == 2) reinterpret_cast<uint16_t*>(orow)[tail0 + tid - 1] = 0;
-            else reinterpret_cast<float*>(orow)[tail0 + tid - 1] = 0.f;
-        }
-    }
-    if (tid == 0) bulk_wait_all<0>();  // the zero buffer must outlive every copy that reads it
-}
-
-// ---- live rows ------------------------------------------------------------------------------------
+// ---- the kernel --------------------------------------------------------------------------------------
 
 template <int DT>
 __global__ void __launch_bounds__(kThreads)
 dlogits_kernel(const void* logits, void* dlogits /* may alias logits */, int64_t ld, int vocab,
                int seq_len, int64_t row0, int64_t n_rows, const int32_t* __restrict__ targets,
-               rapid_stats_t* stats_user, unsigned int* ticket /* zero at launch */, Workspace ws) {
+               rapid_stats_t* stats_user, unsigned int* ticket /* two counters, zero at launch */,
+               unsigned long long stride, int fill_first, Workspace ws) {
     constexpr int ESIZE = (DT == RAPID_BF16) ? 2 : 4;
     constexpr int PER = 16 / ESIZE;  // elements per 16-byte vector
     using RowConst = typename std::conditional<DT == RAPID_BF16, RowConstBf16, RowConstF32>::type;
 
-    extern __shared__ __align__(128) uint8_t ring[];  // kStages x kChunk
+    extern __shared__ __align__(128) uint8_t ring[];  // kStages x kChunk, then kZeroBuf zeros
+    uint8_t* zeros = ring + (size_t)kStages * kChunk;
     __shared__ __align__(8) uint64_t full_bar[kStages];
     __shared__ __align__(8) uint64_t empty_bar[kStages];
     __shared__ int abort_flag;
@@ -115,6 +89,8 @@ dlogits_kernel(const void* logits, void* dlogits /* may alias logits */, int64_t
         abort_flag = 0;
         mbar_init_fence();
     }
+    for (int i = tid; i < kZeroBuf / 16; i += kThreads) reinterpret_cast<uint4*>(zeros)[i] = make_uint4(0, 0, 0, 0);
+    fence_proxy_async_smem();
     __syncthreads();
     volatile int* abortp = &abort_flag;
 
@@ -128,6 +104,28 @@ dlogits_kernel(const void* logits, void* dlogits /* may alias logits */, int64_t
     if (warp == kConsumerWarps) {
         // ------------------------------- producer -------------------------------------------
         if (lane == 0) {
+            const int whole = nvec_row * 16;  // bytes of a row in whole vectors of real columns
+            auto zero_fill = [&](int64_t i) {
+                uint8_t* zrow = static_cast<uint8_t*>(dlogits) + (size_t)i * ld * ESIZE;
+                for (int o = 0; o < whole; o += kZeroBuf) bulk_store(zrow + o, zeros, (uint32_t)min(kZeroBuf, whole - o));
+                bulk_commit();
+                for (int e = nvec_row * PER; e < vocab; ++e) {  // fewer than one vector of columns after them
+                    if (ESIZE == 2) reinterpret_cast<uint16_t*>(zrow)[e] = 0;
+                    else reinterpret_cast<float*>(zrow)[e] = 0.f;
+                }
+                bulk_wait_read<4>();  // a few rows' worth of copies in flight is plenty
+            };
+            // fill_first: the rows without gradient come first, drawn from the second counter, as a pure
+            // write stream; no grid-wide barrier separates the two phases, a CTA goes on to the live rows
+            // as soon as the dead ones have run out.  Otherwise they are filled as they are drawn, between
+            // the loads of the live rows.  (See the launcher for when which.)
+            if (fill_first) {
+                for (;;) {
+                    const unsigned int t = atomicAdd(ticket + 1, 1u);
+                    if ((int64_t)t >= n_rows) break;
+                    if (!row_is_live(ws, row0 + (int64_t)t, seq_len)) zero_fill((int64_t)t);
+                }
+            }
             uint32_t it = 0, j = 0;
             bool ok = true;
             auto stage_free = [&](uint32_t k) {  // the stage that load k goes into has been given back
@@ -135,11 +133,13 @@ dlogits_kernel(const void* logits, void* dlogits /* may alias logits */, int64_t
                 return use == 0 || mbar_wait_bounded(&empty_bar[k % kStages], (use & 1u) ^ 1u, abortp);
             };
             while (ok) {
-                int64_t i;
-                do {  // draw rows until a live one comes, or none is left
-                    i = (int64_t)atomicAdd(ticket, 1u);
-                } while (i < n_rows && !row_is_live(ws, row0 + i, seq_len));
-                if (i >= n_rows) break;
+                const unsigned int t = atomicAdd(ticket, 1u);
+                if ((int64_t)t >= n_rows) break;
+                const int64_t i = (int64_t)(((unsigned long long)t * stride) % (unsigned long long)n_rows);
+                if (!row_is_live(ws, row0 + i, seq_len)) {
+                    if (!fill_first) zero_fill(i);
+                    continue;
+                }
                 const uint8_t* src = static_cast<const uint8_t*>(logits) + (size_t)i * ld * ESIZE;
                 for (int c = 0; c < n_chunks; ++c, ++it) {
                     const int s = it % kStages;
@@ -167,6 +167,7 @@ dlogits_kernel(const void* logits, void* dlogits /* may alias logits */, int64_t
                         if (global_timer_ns() - t0 > kWaitLimitNs) break;
                 }
             }
+            bulk_wait_all<0>();  // the zero buffer must outlive every copy that reads it
         }
     } else {
         // ------------------------------- consumers ------------------------------------------
@@ -249,17 +250,7 @@ template <int DT>
 cudaError_t launch_one(const rapid_desc_t& d, const void* logits_chunk, void* dlogits_chunk,
                        int64_t row0, int64_t n_rows, const int32_t* targets, rapid_stats_t* stats_user,
                        const Workspace& ws, int sm_count, cudaStream_t stream) {
-    constexpr int ESIZE = (DT == RAPID_BF16) ? 2 : 4;
-    // dead rows first: a pure write stream
-    {
-        int64_t grid = (int64_t)sm_count * 16;
-        if (grid > n_rows) grid = n_rows;
-        zero_rows_kernel<ESIZE><<<(unsigned)grid, kZeroThreads, 0, stream>>>(dlogits_chunk, d.ld, d.vocab,
-                                                                             d.seq_len, row0, n_rows, ws);
-        cudaError_t e = cudaGetLastError();
-        if (e != cudaSuccess) return e;
-    }
-    constexpr size_t smem = (size_t)kStages * kChunk;
+    constexpr size_t smem = (size_t)kStages * kChunk + kZeroBuf;
     cudaError_t e = cudaFuncSetAttribute(dlogits_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)smem);
     if (e != cudaSuccess) return e;
@@ -270,10 +261,16 @@ cudaError_t launch_one(const rapid_desc_t& d, const void* logits_chunk, void* dl
     int64_t grid = (int64_t)sm_count * per_sm;
     if (grid > n_rows) grid = n_rows;
     if (n_rows > 0xffffffffll) return cudaErrorInvalidValue;  // the row counter is 32 bits wide
-    e = cudaMemsetAsync(ws.row_ticket, 0, sizeof(unsigned int), stream);
+    e = cudaMemsetAsync(ws.row_ticket, 0, 2 * sizeof(unsigned int), stream);
     if (e != cudaSuccess) return e;
+    // HBM moves more bytes per second when the write-only zero fills come first and the read+write traffic
+    // of the live rows after them than when the two are mixed (64 x 1024 x 151936 bf16 in one launch: 4.83
+    // against 4.92 ms).  A short launch has no time for two ramp-ups, and there filling the dead rows
+    // between the loads wins (64 x 4096 x 32000 fp32 in 16 launches of 2 GB: 7.75 against 8.07 ms).
+    const int fill_first = (double)n_rows * (double)d.vocab * ((DT == RAPID_BF16) ? 2.0 : 4.0) >= 8.0e9 ? 1 : 0;
     dlogits_kernel<DT><<<(unsigned)grid, kThreads, smem, stream>>>(logits_chunk, dlogits_chunk, d.ld, d.vocab, d.seq_len,
-                                                                  row0, n_rows, targets, stats_user, ws.row_ticket, ws);
+                                                                  row0, n_rows, targets, stats_user, ws.row_ticket,
+                                                                  scatter_stride(n_rows), fill_first, ws);
     return cudaGetLastError();
 }
 

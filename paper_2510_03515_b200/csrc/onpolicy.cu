@@ -759,22 +759,6 @@ onpolicy_loss_kernel(int n_seq, float* __restrict__ loss_out, rapid_stats_t* __r
 
 }  // namespace
 
-// A multiplier coprime to n and near 0.62 n: t -> (t * stride) mod n visits every row once, neighbours in t far apart.
-static unsigned long long scatter_stride(int64_t n) {
-    auto gcd = [](unsigned long long a, unsigned long long b) {
-        while (b) {
-            const unsigned long long c = a % b;
-            a = b;
-            b = c;
-        }
-        return a;
-    };
-    unsigned long long s = (unsigned long long)((double)n * 0.6180339887498949);
-    if (s < 1) s = 1;
-    while (gcd(s, (unsigned long long)n) != 1) ++s;
-    return s;
-}
-
 cudaError_t launch_onpolicy(const rapid_desc_t& d, const void* logits, void* dlogits, const int32_t* targets,
                             const uint8_t* mask, const float* rewards, const int32_t* group_offsets, float* loss,
                             float* token_logp, float* adv, rapid_stats_t* stats, const Workspace& ws, int sm_count,

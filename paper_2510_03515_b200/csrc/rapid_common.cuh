@@ -34,7 +34,7 @@ struct Workspace {
     int32_t* seq_tokens;    // [N]
     int32_t* seq_bad;       // [N] rows with a target id outside [0, V)
     rapid_stats_t* stats;   // [1]
-    unsigned int* row_ticket;  // [1] next row of the statistics pass (zeroed by each launch)
+    unsigned int* row_ticket;  // [2] row counters of the streaming kernels (zeroed by each launch)
 };
 
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -65,7 +65,7 @@ __host__ inline size_t carve_workspace(const rapid_desc_t& d, void* base, Worksp
     ws.seq_tokens = reinterpret_cast<int32_t*>(take(N * 4));
     ws.seq_bad = reinterpret_cast<int32_t*>(take(N * 4));
     ws.stats = reinterpret_cast<rapid_stats_t*>(take(sizeof(rapid_stats_t)));
-    ws.row_ticket = reinterpret_cast<unsigned int*>(take(sizeof(unsigned int)));
+    ws.row_ticket = reinterpret_cast<unsigned int*>(take(2 * sizeof(unsigned int)));
     if (w) *w = ws;
     return off;
 }
@@ -148,6 +148,25 @@ __device__ __forceinline__ int warp_sum(int v) {
 }
 
 #endif  // __CUDACC__
+
+// Rows are handed to CTAs through a counter; draw t stands for row (t * stride) mod n.  The stride is coprime
+// to n (every row is visited once) and near 0.62 n, so that rows drawn at about the same time lie far apart:
+// the memory system then sees the batch's average mix of rows that are read and written and rows that are
+// only zero-filled, rather than one kind after the other (masked rows cluster at the end of every generation).
+inline unsigned long long scatter_stride(int64_t n) {
+    auto gcd = [](unsigned long long a, unsigned long long b) {
+        while (b) {
+            const unsigned long long c = a % b;
+            a = b;
+            b = c;
+        }
+        return a;
+    };
+    unsigned long long s = (unsigned long long)((double)n * 0.6180339887498949);
+    if (s < 1) s = 1;
+    while (gcd(s, (unsigned long long)n) != 1) ++s;
+    return s;
+}
 
 // Host-side launchers (each enqueues on `stream` and returns the launch status).
 cudaError_t launch_row_stats(const rapid_desc_t& d, const void* logits_chunk, int64_t row0,
