@@ -343,14 +343,14 @@ def mean_median(xs):
 # DRAM traffic per algorithmic byte, from the ncu captures summarised under profiles/ (counters
 # dram__bytes_read.sum + dram__bytes_write.sum of a smaller launch of the same kernel; traffic grows
 # in proportion to the rows processed).  NOT counters of this run: the line says so.
-TRAFFIC_P2_PER_BYTE = 0.9719
+TRAFFIC_P2_PER_BYTE = 0.9873
 TRAFFIC_P2_SOURCE = "profiles/logits_in_path_slm_bf16.md: ncu dram bytes of a 2.5 GB launch x rows of this one"
 # the on-policy kernel: dram__bytes_read.sum per byte of live rows, dram__bytes_write.sum per byte of all rows
-TRAFFIC_OP_READ_PER_LIVE_BYTE = 1.288
-TRAFFIC_OP_WRITE_PER_ROW_BYTE = 0.977
+TRAFFIC_OP_READ_PER_LIVE_BYTE = 1.280
+TRAFFIC_OP_WRITE_PER_ROW_BYTE = 0.978
 TRAFFIC_OP_SOURCE = "profiles/onpolicy_rows_kernel_slm_bf16.md: ncu dram bytes of an 8192-row launch x rows of this one"
 # pass 1's secondary ceiling: share of cycles the MUFU (ex2) pipe is busy, same captures
-MUFU_PIPE_PCT_PASS1 = 80.2
+MUFU_PIPE_PCT_PASS1 = 81.1
 MUFU_SOURCE = "profiles/logits_in_path_slm_bf16.md (ncu pipe utilisation of row_stats_kernel)"
 
 
@@ -458,7 +458,7 @@ def run_ours(args, rk: Rank):
                      "frac_of_8TBs_nominal": ach_p2 / 8000.0, "ms_per_launch": p2 / n_chunks,
                      "ms_per_step": p2, "ms_per_step_median": p2_med,
                      "achieved_at_median": bytes_p2 / (p2_med * 1e-3) / 1e9,
-                     "algorithmic_bytes_per_launch": bytes_p2 / n_chunks, "launches_per_step": 2 * n_chunks,
+                     "algorithmic_bytes_per_launch": bytes_p2 / n_chunks, "launches_per_step": n_chunks,
                      "traffic": (TRAFFIC_P2_PER_BYTE * bytes_p2) if name == "slm" else None,
                      "traffic_source": TRAFFIC_P2_SOURCE if name == "slm" else None},
         "roofline_pass1": {"bound": "hbm", "kernel": "row_stats_kernel (pass 1)", "achieved": ach_p1,
