@@ -839,6 +839,16 @@ def run_extras(args, rk: Rank) -> dict:
             r["pass1"] = ln["roofline_pass1"]
             r["step"] = ln["roofline_step"]
         out[key] = r
+    # the oracle on a bounded slice of the two configurations that have no timed GPU run of their own
+    # (tiny: launch-bound, parity only; stale: the shape class of slm), so that every configuration has one
+    if rk.rank == 0 and not args.skip_cpu:
+        other = {}
+        for name in ("tiny", "stale"):
+            c = oracle_sample(synth.CONFIGS[name], target_seconds=3.0, single_thread=False)
+            for k in ("seconds", "tokens", "single_thread"):
+                c.pop(k, None)
+            other[name] = c
+        out["cpu_baseline_other_configs"] = other
     return out
 
 
