@@ -559,18 +559,25 @@ def run_e2e(rb, args, desc, w, logits, tok, behav, dlogits, ws, loss, token_logp
            "d2h_bytes_per_step": 4, "steps": steps, "ms_per_step": ms / steps, "host_buffer": mode,
            "d2h_is": "the loss", "result_left_on_device_bytes": int(nbytes),
            "result_left_on_device": "dlogits (consumed on the device by the backward pass of the model)"}
+    # the second figure needs a second pinned buffer on every rank: each rank tries, all agree, then all
+    # time it or none does (a rank that skipped the timed loop would leave the others at its barrier)
     out_grad = None
+    why = ""
     try:
-        enough = psutil.virtual_memory().available > 2 * nbytes
-        enough = bool(rk.sum_over_ranks(0.0 if enough else 1.0) == 0.0)      # every rank, or none
-        if enough:
+        if psutil.virtual_memory().available > 2 * nbytes:
             host_grad = torch.empty(logits.shape, dtype=logits.dtype, pin_memory=True)
-            ms2 = timed()
-            out_grad = {"value": tokens * steps / (ms2 * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
-                        "d2h_bytes_per_step": int(nbytes) + 4, "steps": steps, "ms_per_step": ms2 / steps,
-                        "d2h_is": "the loss and all of dlogits"}
-    except RuntimeError as ex:          # pinning the second buffer failed: report why, keep the first figure
-        out_grad = {"unavailable": str(ex).splitlines()[0][:200]}
+        else:
+            why = "not enough host memory for a second pinned buffer"
+    except RuntimeError as ex:
+        host_grad, why = None, str(ex).splitlines()[0][:200]
+    if rk.sum_over_ranks(0.0 if host_grad is not None else 1.0) == 0.0:
+        ms2 = timed()
+        out_grad = {"value": tokens * steps / (ms2 * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+                    "d2h_bytes_per_step": int(nbytes) + 4, "steps": steps, "ms_per_step": ms2 / steps,
+                    "d2h_is": "the loss and all of dlogits"}
+    else:
+        host_grad = None
+        out_grad = {"unavailable": why or "another rank could not pin its buffer"}
     del d_logits, host_logits, host_grad
     return out, out_grad
 
