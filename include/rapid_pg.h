@@ -148,11 +148,13 @@ const char* rapid_status_string(rapid_status_t status);
 int32_t rapid_version(void);
 
 /*
- * Size of the scratch workspace the logits-in calls need for `desc` (16 bytes per row plus a
+ * Size of the scratch workspace the logits-in calls need for `desc` (21 bytes per row plus a
  * few per generation).  `bytes` is host memory.  The workspace must be 256-byte aligned device
  * memory; its contents need not be initialised.  Between rapid_pg_stats_chunk, rapid_pg_finalize
  * and rapid_pg_dlogits_chunk it carries the per-row and per-generation state and must not be
- * touched by the caller.
+ * touched by the caller.  It also holds the counters from which the streaming kernels draw their
+ * rows, so calls that use the same workspace must not overlap on the device: put them on one
+ * stream, or order them with events (the blocks of the chunked form included).
  */
 rapid_status_t rapid_workspace_bytes(const rapid_desc_t* desc, size_t* bytes);
 
