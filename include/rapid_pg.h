@@ -98,7 +98,12 @@ enum {
     /* long-K ones (dhidden, dW) on single CTAs, the mix measured fastest; these two flags force     */
     /* all four one way (CTA_PAIRS wins if both are given).                                          */
     RAPID_FLAG_HEAD_CTA_PAIRS = 128u,
-    RAPID_FLAG_HEAD_SINGLE_CTA = 256u
+    RAPID_FLAG_HEAD_SINGLE_CTA = 256u,
+    /* rapid_pg_loss_fused_head only: dW is written as bf16 ([D, ld] bf16, same pitch rule as w_vocab) */
+    /* instead of float: half the bytes, for a weight gradient that a bf16 optimizer state consumes.  */
+    /* The float accumulator is rounded once per backward chunk of 16384 rows; with more rows than    */
+    /* that the chunks' contributions are added in bf16, one rounding per chunk.                      */
+    RAPID_FLAG_HEAD_DW_BF16 = 512u
 };
 
 /* Problem descriptor (host memory, plain data, 48 bytes). */
@@ -349,9 +354,10 @@ rapid_status_t rapid_pg_loss_onpolicy_fwd_bwd(const rapid_desc_t* desc, const vo
  *   targets, mask, behav_logp, rewards, group_offsets: as for rapid_pg_loss_fwd_bwd
  *   loss        [1] float out
  *   dhidden     [T, D] bf16 out (pitch D); rows that are masked or have g_n = 0 come out as zeros
- *   dW          [D, ld] float out.  Stores go out in 16-byte units: when vocab is not a multiple
- *               of 4, the columns from vocab up to the next multiple of 4 are written as zeros;
- *               columns beyond that are untouched
+ *   dW          [D, ld] float out ([D, ld] bf16 with RAPID_FLAG_HEAD_DW_BF16).  Stores go out in
+ *               16-byte units: when vocab is not a multiple of 4 (of 8 for bf16), the columns from
+ *               vocab up to the next such multiple are written as zeros; columns beyond that are
+ *               untouched
  *   token_logp, adv, stats: optional outputs as for rapid_pg_loss_fwd_bwd
  *   workspace   rapid_fused_head_workspace_bytes(desc, hidden_dim) bytes, 1024-byte aligned.  It
  *               holds, besides the per-row state, two floats per row per 256 vocabulary columns

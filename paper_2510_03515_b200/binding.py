@@ -37,6 +37,7 @@ FLAG_NORM_GIVEN = 32
 FLAG_HEAD_STORE_LOGITS = 64
 FLAG_HEAD_CTA_PAIRS = 128
 FLAG_HEAD_SINGLE_CTA = 256
+FLAG_HEAD_DW_BF16 = 512
 
 # every symbol declared in include/rapid_pg.h
 EXPORTS = (

@@ -364,10 +364,11 @@ struct DzStore {
 
 // ---- backward epilogues 2 and 3: plain stores ------------------------------------------------------------
 
-struct StoreBf16 {  // dh
+struct StoreBf16 {  // dh; dW when the caller wants it in bf16
     struct Params {
         CUtensorMap map;  // [M, N] bf16, box 64 x 32
         int N;
+        int accumulate;   // add to what is there (dW, second and later row chunks) instead of overwriting
     };
     const Params& p;
     const int quarter, lane;
@@ -392,7 +393,7 @@ struct StoreBf16 {  // dh
                     *reinterpret_cast<uint4*>(buf + swz128(lane, half * 4 + k)) = make_uint4(o[0], o[1], o[2], o[3]);
                 }
             }
-            st.commit(&p.map, buf, n0 + q * 64, m0 + quarter * 32);
+            st.commit(&p.map, buf, n0 + q * 64, m0 + quarter * 32, p.accumulate != 0);
         }
     }
     __device__ void finish() { st.finish(); }
@@ -516,6 +517,7 @@ extern "C" rapid_status_t rapid_pg_loss_fused_head(
     const uint32_t pair_mask = (desc->flags & RAPID_FLAG_HEAD_CTA_PAIRS) ? 15u
                                : (desc->flags & RAPID_FLAG_HEAD_SINGLE_CTA) ? 0u : 3u;
     const bool pairs = (pair_mask & 4u) != 0;
+    const bool dw_bf16 = (desc->flags & RAPID_FLAG_HEAD_DW_BF16) != 0;  // dW is [D, ld] bf16 instead of float
     CUtensorMap w_k_half;  // B of dh for a CTA of a pair: 128 of the tile's 256 rows of W^T per box
     if (pairs && !make_map_bf16(&w_k_half, w_vocab, D, V, ld, BK, BN / 2)) return RAPID_ERR_CUDA;
 
@@ -566,12 +568,14 @@ extern "C" rapid_status_t rapid_pg_loss_fused_head(
         DzStore::Params dzp;
         StoreBf16::Params dhp;
         StoreF32::Params dwp;
+        StoreBf16::Params dwp16;
         ok = make_map_bf16(&hc_k, h_c, R, D, D, BK, BM)                // A of recompute: rows x K
              && make_map_bf16(&hc_mn, h_c, R, D, D, 64, BK)            // A of dW: K(=rows) x M(=D)
              && make_map_bf16(&dz_k, dz_c, R, V, hs.ldz, BK, BM)      // A of dh: rows x K(=V)
              && make_map_bf16(&dz_mn, dz_c, R, V, hs.ldz, 64, BK)     // B of dW: K(=rows) x N(=V)
              && make_map_bf16(&dzp.map, dz_c, R, V, hs.ldz, 64, 32)   // stores
-             && make_map_bf16(&dhp.map, dh_c, R, D, D, 64, 32) && make_map_f32(&dwp.map, dW, D, V, ld, 32, 32);
+             && make_map_bf16(&dhp.map, dh_c, R, D, D, 64, 32)
+             && (dw_bf16 ? make_map_bf16(&dwp16.map, dW, D, V, ld, 64, 32) : make_map_f32(&dwp.map, dW, D, V, ld, 32, 32));
         if (!ok) return RAPID_ERR_CUDA;
         const int mR = (int)((R + BM - 1) / BM);
 
@@ -590,17 +594,23 @@ extern "C" rapid_status_t rapid_pg_loss_fused_head(
             return RAPID_ERR_CUDA;
 
         dhp.N = D;
+        dhp.accumulate = 0;
         Shape sdh{mR, (D + BN - 1) / BN, (V + BK - 1) / BK, N_FASTEST};
         if (((pair_mask & 4u) ? launch_gemm_pair<StoreBf16, false, false>(dz_k, w_k_half, sdh, sms, hs.status, dhp, st)
                    : launch_gemm<StoreBf16, false, false>(dz_k, w_k, sdh, sms, hs.status, dhp, st)) != cudaSuccess)
             return RAPID_ERR_CUDA;
 
-        dwp.N = V;
-        dwp.accumulate = (r0 > 0) ? 1 : 0;
+        dwp.N = dwp16.N = V;
+        dwp.accumulate = dwp16.accumulate = (r0 > 0) ? 1 : 0;
         Shape sdw{(D + BM - 1) / BM, nV, (int)((R + BK - 1) / BK), M_FASTEST};
-        if (((pair_mask & 8u) ? launch_gemm_pair<StoreF32, true, true>(hc_mn, dz_mn, sdw, sms, hs.status, dwp, st)
-                   : launch_gemm<StoreF32, true, true>(hc_mn, dz_mn, sdw, sms, hs.status, dwp, st)) != cudaSuccess)
-            return RAPID_ERR_CUDA;
+        cudaError_t ew;
+        if (dw_bf16)
+            ew = (pair_mask & 8u) ? launch_gemm_pair<StoreBf16, true, true>(hc_mn, dz_mn, sdw, sms, hs.status, dwp16, st)
+                                  : launch_gemm<StoreBf16, true, true>(hc_mn, dz_mn, sdw, sms, hs.status, dwp16, st);
+        else
+            ew = (pair_mask & 8u) ? launch_gemm_pair<StoreF32, true, true>(hc_mn, dz_mn, sdw, sms, hs.status, dwp, st)
+                                  : launch_gemm<StoreF32, true, true>(hc_mn, dz_mn, sdw, sms, hs.status, dwp, st);
+        if (ew != cudaSuccess) return RAPID_ERR_CUDA;
     }
 
     publish_status_kernel<<<1, 1, 0, st>>>(hs.status, stats, ws.stats);

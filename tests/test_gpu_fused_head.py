@@ -92,7 +92,8 @@ def run_head(b, w, behav, ld_pad=0, eta=2.0, flags=0):
     ws = rb.alloc_fused_head_workspace(desc, D, dev)
     loss = torch.full((1,), float("nan"), device=dev)
     dh = torch.full((T + 2, D), 7.0, dtype=torch.bfloat16, device=dev)   # one guard row on each side
-    dW = torch.full((D + 2, ld), 5.0, dtype=torch.float32, device=dev)
+    dw_bf16 = bool(flags & rb.FLAG_HEAD_DW_BF16)
+    dW = torch.full((D + 2, ld), 5.0, dtype=torch.bfloat16 if dw_bf16 else torch.float32, device=dev)
     tl = torch.full((T,), float("nan"), device=dev)
     adv = torch.full((w.n_seq,), float("nan"), device=dev)
     stats = rb.alloc_stats(dev)
@@ -103,11 +104,13 @@ def run_head(b, w, behav, ld_pad=0, eta=2.0, flags=0):
     assert torch.all(dh[0] == 7.0) and torch.all(dh[T + 1] == 7.0), "dhidden guard rows overwritten"
     assert torch.all(dW[0] == 5.0) and torch.all(dW[D + 1] == 5.0), "dW guard rows overwritten"
     if ld_pad:
-        v4 = (V + 3) // 4 * 4   # stores go out in 16-byte units: up to 3 pad columns become zero
+        unit = 8 if dw_bf16 else 4
+        v4 = (V + unit - 1) // unit * unit   # stores go out in 16-byte units: the pad columns of the last unit become zero
         assert torch.all(dW[1:D + 1, v4:] == 5.0), "dW columns beyond the 16-byte unit overwritten"
         assert torch.all((dW[1:D + 1, V:v4] == 5.0) | (dW[1:D + 1, V:v4] == 0.0))
     return {"loss": loss.item(), "dh": dh[1:T + 1].float().cpu().numpy().astype(np.float64),
-            "dW": dW[1:D + 1, :V].cpu().numpy().astype(np.float64), "token_logp": tl.cpu().numpy(),
+            "dW": dW[1:D + 1, :V].float().cpu().numpy().astype(np.float64), "dw_bf16": dw_bf16,
+            "token_logp": tl.cpu().numpy(),
             "adv": adv.cpu().numpy(), "stats": rb.read_stats(stats)}
 
 
@@ -129,6 +132,11 @@ def compare_head(o, g, w):
                           f"{(np.abs(g['dh'] - o['dh']) / tol_h).max():.2f}"
     rss_w = np.sqrt((o["h"] ** 2).T @ (o["dz"] ** 2))
     tol_w = 2.0 ** -6 * rss_w + 1e-6 * np.abs(o["dW"]) + 1e-12
+    if g.get("dw_bf16"):
+        # dW itself rounded to bf16: once per backward chunk of 16384 rows (2^-8 relative each), and
+        # the chunks' sums are added in bf16
+        n_chunks = (w.n_rows + 16383) // 16384
+        tol_w = tol_w + (2 * n_chunks - 1) * 2.0 ** -8 * np.abs(o["dW"]) + (n_chunks - 1) * 2.0 ** -8 * np.abs(o["h"]).T @ np.abs(o["dz"])
     bad = np.abs(g["dW"] - o["dW"]) > tol_w
     assert not bad.any(), f"dW: {bad.sum()} elements out of tolerance, worst ratio " \
                           f"{(np.abs(g['dW'] - o['dW']) / tol_w).max():.2f}"
@@ -210,6 +218,31 @@ def test_fused_head_cta_pairs(V, D, L, pad, extra):
     o = oracle_head(b, w, flags=extra)
     g = run_head(b, w, o["behav"], ld_pad=pad, flags=extra | rb.FLAG_HEAD_CTA_PAIRS)
     compare_head(o, g, w)
+
+
+@pytest.mark.parametrize("extra", [0, rb.FLAG_HEAD_CTA_PAIRS, rb.FLAG_HEAD_STORE_LOGITS])
+@pytest.mark.parametrize("V,D,L,pad", [(1000, 192, 40, 0), (777, 200, 50, 7), (40, 8, 3, 0)])
+def test_fused_head_weight_gradient_in_bf16(V, D, L, pad, extra):
+    """RAPID_FLAG_HEAD_DW_BF16: dW comes out as bf16 (guard rows and pad columns untouched), through the
+    single-CTA and the CTA-pair kernels."""
+    pad = (-V) % 8 + pad if (V + pad) % 8 else pad
+    w = synth.CONFIGS["fused"].scaled(n_prompts=3, group_size=4, seq_len=L, vocab=V, hidden=D,
+                                      length_mode="uniform", len_lo=max(1, L // 3), reward_mode="per_prompt_const",
+                                      seed=300 + V)
+    b = synth.make_head(w)
+    o = oracle_head(b, w, flags=extra & rb.FLAG_HEAD_STORE_LOGITS)
+    g = run_head(b, w, o["behav"], ld_pad=pad, flags=extra | rb.FLAG_HEAD_DW_BF16)
+    compare_head(o, g, w)
+
+
+def test_fused_head_weight_gradient_in_bf16_over_two_backward_chunks():
+    """18000 rows: the second chunk's contribution is added to a bf16 dW."""
+    w = synth.CONFIGS["fused"].scaled(n_prompts=3, group_size=3, seq_len=2000, vocab=600, hidden=64,
+                                      length_mode="uniform", len_lo=1500, reward_mode="per_prompt", seed=71)
+    b = synth.make_head(w)
+    b["rewards"] = torch.randn(w.n_seq, generator=torch.Generator().manual_seed(8))
+    o = oracle_head(b, w)
+    compare_head(o, run_head(b, w, o["behav"], flags=rb.FLAG_HEAD_DW_BF16), w)
 
 
 def test_fused_head_cta_pairs_many_tiles_and_two_backward_chunks():
