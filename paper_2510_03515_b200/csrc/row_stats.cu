@@ -62,16 +62,17 @@ struct FloatSum {
 //    1.3e-8 relative, which shifts the log-sum-exp by that times the softmax-weighted mean distance
 //    below the shift: 5e-8 for these logits.
 //  * the hardware exponential's relative error on negative arguments, averaged over the fraction of
-//    the argument, is kEx2Bias (measured over all 2^23 fractions on sm_100a: -5.0e-8, the same to 3 %
-//    for every integer part; errors lie in [-1.44e-7, +0.63e-7]); a sum of many terms carries that
-//    mean, and is divided by 1 + kEx2Bias.  bf16 logits take few distinct values, so with a common
+//    the argument, is kEx2Bias (measured over all 2^23 fractions on sm_100a: -4.95e-8 for arguments in
+//    [-1, 0), -4.97e-8 in [-2, -1), -5.02e-8 in [-5, -4), -5.11e-8 in [-20, -19); the terms that carry a
+//    row's mass lie within a few units of the shift; errors lie in [-1.44e-7, +0.63e-7]); a sum of many
+//    terms carries that mean, and is divided by 1 + kEx2Bias.  bf16 logits take few distinct values, so with a common
 //    integer shift the fraction of x_v would depend on z_v alone and the sum would carry the errors of
 //    those few fractions (1e-8 either way) instead of the mean; the 16-bit fraction `off`, different
 //    for every thread, spreads each logit value over 128 fractions.
 //  * the thread's largest logit, which may carry nearly all of the row's probability, gets no such
 //    statistical treatment: its hardware exponential is taken out of S again at the end of the sweep
 //    and replaced by the exact value in double.
-constexpr float kEx2Bias = -5.0e-8f;
+constexpr float kEx2Bias = -4.95e-8f;
 constexpr float kK1 = 47274.f / 32768.f;                   // log2(e) rounded down to 16 bits
 constexpr float kK2 = (float)(kLog2eD - 47274.0 / 32768.0);  // > 0, so that -inf logits stay -inf
 
@@ -96,7 +97,11 @@ __device__ __forceinline__ void bf16_batch(const uint4 (&q)[U], float off, float
     // a pair of logits at a time in the packed two-float forms (one instruction for two multiply-adds
     // or two additions, each rounded like its scalar form)
     const uint64_t k1 = f32x2(kK1, kK1), k2 = f32x2(kK2, kK2), nsh2 = f32x2(-sh, -sh);
-    uint64_t s2 = f32x2(0.f, 0.f);
+    // eight partial sums of at most U terms each (four packed pairs, one per word of a vector): a float
+    // partial that holds one of the row's largest terms drops every later addend below half an ulp of
+    // it, and the fewer addends share a partial with such a term, the less is lost (with two partials of
+    // 32 terms that loss was the largest bias left, 2e-9 on N(0,3) logits)
+    uint64_t s2[4] = {f32x2(0.f, 0.f), f32x2(0.f, 0.f), f32x2(0.f, 0.f), f32x2(0.f, 0.f)};
 #pragma unroll
     for (int j = 0; j < U; ++j) {
         const uint32_t w[4] = {q[j].x, q[j].y, q[j].z, q[j].w};
@@ -105,11 +110,11 @@ __device__ __forceinline__ void bf16_batch(const uint4 (&q)[U], float off, float
             const uint64_t z2 = f32x2(bf16_lo(w[k]), bf16_hi(w[k]));
             float x0, x1;
             f32x2_split(f32x2_fma(z2, k2, f32x2_fma(z2, k1, nsh2)), x0, x1);
-            s2 = f32x2_add(s2, f32x2(ex2_approx(x0), ex2_approx(x1)));
+            s2[k] = f32x2_add(s2[k], f32x2(ex2_approx(x0), ex2_approx(x1)));
         }
     }
     float s0, s1;
-    f32x2_split(s2, s0, s1);
+    f32x2_split(f32x2_add(f32x2_add(s2[0], s2[1]), f32x2_add(s2[2], s2[3])), s0, s1);
     const float b = s0 + s1;
     if (b > S.s) {  // keep the larger operand first, as Fast2Sum wants (early batches only)
         const float old = S.s;
